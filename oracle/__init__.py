@@ -1,0 +1,120 @@
+"""CPU oracle for the emulated collectives -- TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package.  It does not import the CUDA package and shares nothing with it.
+
+``nuna_oracle.c`` is the plain definition (bf16 storage, binary32 fold in rank
+order, one final round to nearest even); this module compiles it with gcc and
+exposes it over numpy ``uint16`` arrays.  ``exact_model`` is a second, exact
+rational-arithmetic model used to pin the C code on small inputs, and
+``nap_planner`` restates the paper's placement algorithm (Algorithm 1).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import List, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "nuna_oracle.c")
+_LIB = os.path.join(_HERE, "libnuna_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle (gcc, -O2, strict IEEE: no fast-math) and return the library path."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    cmd = ["gcc", "-O2", "-std=c11", "-fno-fast-math", "-ffp-contract=off", "-fopenmp",
+           "-fPIC", "-shared", "-Wall", "-Wextra", "-o", tmp, _SRC]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        pp = ctypes.POINTER(ctypes.c_void_p)
+        for name in ("nuna_oracle_allreduce_bf16", "nuna_oracle_reduce_scatter_bf16",
+                     "nuna_oracle_allgather_bf16"):
+            fn = getattr(lib, name)
+            fn.argtypes = [pp, pp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int]
+            fn.restype = None
+        lib.nuna_oracle_fold_bf16.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        lib.nuna_oracle_fold_bf16.restype = ctypes.c_uint16
+        lib.nuna_oracle_rne_bf16.argtypes = [ctypes.c_float]
+        lib.nuna_oracle_rne_bf16.restype = ctypes.c_uint16
+        lib.nuna_oracle_widen_bf16.argtypes = [ctypes.c_uint16]
+        lib.nuna_oracle_widen_bf16.restype = ctypes.c_float
+        _lib = lib
+    return _lib
+
+
+def _ptrs(arrs: Sequence[np.ndarray]):
+    tab = (ctypes.c_void_p * len(arrs))()
+    for i, a in enumerate(arrs):
+        assert a.dtype == np.uint16 and a.flags.c_contiguous
+        tab[i] = a.ctypes.data
+    return tab
+
+
+def _check_src(src: Sequence[np.ndarray], length: int):
+    if len(src) < 1:
+        raise ValueError("need at least one rank")
+    for a in src:
+        if a.dtype != np.uint16 or a.ndim != 1 or len(a) != length:
+            raise ValueError("every rank buffer must be a 1-D uint16 array of the same length")
+
+
+def allreduce(src: Sequence[np.ndarray], nthreads: int = 1) -> List[np.ndarray]:
+    """One result array per destination rank (all equal by definition)."""
+    n, count = len(src), len(src[0])
+    _check_src(src, count)
+    src = [np.ascontiguousarray(a) for a in src]
+    dst = [np.empty(count, dtype=np.uint16) for _ in range(n)]
+    _load().nuna_oracle_allreduce_bf16(_ptrs(src), _ptrs(dst), n, count, int(nthreads))
+    return dst
+
+
+def reduce_scatter(src: Sequence[np.ndarray], nthreads: int = 1) -> List[np.ndarray]:
+    """``src[k]`` holds ``N*S`` elements; returns N arrays of S elements."""
+    n, total = len(src), len(src[0])
+    _check_src(src, total)
+    if total % n:
+        raise ValueError("source length must be a multiple of the rank count")
+    shard = total // n
+    src = [np.ascontiguousarray(a) for a in src]
+    dst = [np.empty(shard, dtype=np.uint16) for _ in range(n)]
+    _load().nuna_oracle_reduce_scatter_bf16(_ptrs(src), _ptrs(dst), n, shard, int(nthreads))
+    return dst
+
+
+def allgather(src: Sequence[np.ndarray], nthreads: int = 1) -> List[np.ndarray]:
+    """``src[r]`` holds S elements; returns N arrays of ``N*S`` elements."""
+    n, shard = len(src), len(src[0])
+    _check_src(src, shard)
+    src = [np.ascontiguousarray(a) for a in src]
+    dst = [np.empty(n * shard, dtype=np.uint16) for _ in range(n)]
+    _load().nuna_oracle_allgather_bf16(_ptrs(src), _ptrs(dst), n, shard, int(nthreads))
+    return dst
+
+
+def fold(vals) -> int:
+    """Rank-ordered sum of one column of bf16 patterns."""
+    a = np.ascontiguousarray(np.asarray(vals, dtype=np.uint16))
+    return int(_load().nuna_oracle_fold_bf16(a.ctypes.data, len(a)))
+
+
+def rne_bf16(x: float) -> int:
+    return int(_load().nuna_oracle_rne_bf16(x))
+
+
+def widen_bf16(h: int) -> float:
+    return float(_load().nuna_oracle_widen_bf16(h))

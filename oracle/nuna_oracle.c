@@ -1,0 +1,115 @@
+/*
+ * CPU oracle for the emulated collectives.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the slow, plain definition that the CUDA library is checked
+ * against.  It shares no code, header, table or helper with the CUDA path and
+ * is called only by the tests, by the smoke check and by the benchmark's CPU
+ * baseline leg.  Nothing on the product path may call it.
+ *
+ * What it computes.  The paper describes the collectives only at the level of
+ * their meaning (Section 2.1: allreduce aggregates the partial activations of
+ * all ranks, allgather assembles every rank's chunk in every rank's output;
+ * Figure "Allocation_Diagram": allgather as local load + remote store of each
+ * rank's chunk into every rank's buffer; Section 5.1: the direct / all-pairs
+ * algorithm).  The numerics are fixed by this build's problem statement:
+ * bf16 storage, binary32 accumulation in fixed rank order 0..N-1, one final
+ * round-to-nearest-even to bf16, the same value in every destination.
+ *
+ *   f(h)   : bf16 pattern h  ->  binary32 whose bits are h << 16        (exact)
+ *   rne(x) : binary32 -> bf16, round to nearest, ties to even; NaN -> 0x7FFF
+ *   allreduce      dst[d][i]       = rne((((f(src[0][i]) + f(src[1][i])) + ...) + f(src[N-1][i])))
+ *   reduce_scatter dst[r][j]       = the same fold over src[0..N-1][r*S + j]
+ *   allgather      dst[d][r*S + j] = src[r][j]                          (16-bit copy)
+ *
+ * The accumulator starts from f(src[0][i]), not from +0, so N values take N-1
+ * additions and an all-(-0) column stays -0.  Every partial sum is a binary32
+ * (SSE scalar add on x86-64: no extended precision, default rounding, no
+ * flush-to-zero).  Compile without -ffast-math.
+ *
+ * Parity pins: see tests/test_oracle_pins.py (closed forms on exactly
+ * representable integers, order / rounding / signed-zero / subnormal /
+ * overflow pins, an exact-rational second model, brute force on tiny inputs).
+ */
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+
+static float bf16_to_f32(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float x;
+    memcpy(&x, &u, sizeof x);
+    return x;
+}
+
+static uint16_t f32_to_bf16_rne(float x)
+{
+    uint32_t u;
+    memcpy(&u, &x, sizeof u);
+    if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu) != 0u)
+        return 0x7FFFu;                              /* NaN: canonical quiet NaN */
+    /* Add half of the dropped field, minus one when the kept LSB is even, so a
+       tie moves to the even neighbour.  A carry may run into the exponent,
+       which is how the largest finite values round up to infinity. */
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+/* Fold one column: the n values of one element index, in rank order. */
+uint16_t nuna_oracle_fold_bf16(const uint16_t *vals, int n)
+{
+    volatile float acc = bf16_to_f32(vals[0]);       /* volatile: each partial sum is stored as binary32 */
+    for (int r = 1; r < n; ++r)
+        acc = acc + bf16_to_f32(vals[r]);
+    return f32_to_bf16_rne(acc);
+}
+
+static uint16_t fold_column(const uint16_t *const *src, int nranks, size_t i)
+{
+    float acc = bf16_to_f32(src[0][i]);
+    for (int r = 1; r < nranks; ++r)
+        acc = acc + bf16_to_f32(src[r][i]);
+    return f32_to_bf16_rne(acc);
+}
+
+/* allreduce: every dst[d] (count elements) receives the rank-ordered sum. */
+void nuna_oracle_allreduce_bf16(const uint16_t *const *src, uint16_t *const *dst,
+                                int nranks, size_t count, int nthreads)
+{
+    (void)nthreads;
+#pragma omp parallel for schedule(static) num_threads(nthreads) if (nthreads > 1)
+    for (size_t i = 0; i < count; ++i) {
+        uint16_t out = fold_column(src, nranks, i);
+        for (int d = 0; d < nranks; ++d)
+            dst[d][i] = out;
+    }
+}
+
+/* reduce_scatter: src[k] has nranks*shard elements, dst[r] has shard elements. */
+void nuna_oracle_reduce_scatter_bf16(const uint16_t *const *src, uint16_t *const *dst,
+                                     int nranks, size_t shard, int nthreads)
+{
+    (void)nthreads;
+    for (int r = 0; r < nranks; ++r) {
+#pragma omp parallel for schedule(static) num_threads(nthreads) if (nthreads > 1)
+        for (size_t j = 0; j < shard; ++j)
+            dst[r][j] = fold_column(src, nranks, (size_t)r * shard + j);
+    }
+}
+
+/* allgather: src[r] has shard elements, every dst[d] has nranks*shard elements. */
+void nuna_oracle_allgather_bf16(const uint16_t *const *src, uint16_t *const *dst,
+                                int nranks, size_t shard, int nthreads)
+{
+    (void)nthreads;
+    for (int d = 0; d < nranks; ++d)
+        for (int r = 0; r < nranks; ++r) {
+#pragma omp parallel for schedule(static) num_threads(nthreads) if (nthreads > 1)
+            for (size_t j = 0; j < shard; ++j)
+                dst[d][(size_t)r * shard + j] = src[r][j];
+        }
+}
+
+/* The two conversions on their own, so the tests can pin them separately. */
+uint16_t nuna_oracle_rne_bf16(float x) { return f32_to_bf16_rne(x); }
+float nuna_oracle_widen_bf16(uint16_t h) { return bf16_to_f32(h); }
