@@ -1,0 +1,126 @@
+/*
+ * nuna.h -- C ABI of the B200 (sm_100a) emulated-rank collective library.
+ *
+ * N ranks are emulated as N separate device buffers on ONE GPU.  Every
+ * collective reads N "rank" source buffers and writes N "rank" destination
+ * buffers; there is no inter-GPU traffic.  The operations are those the paper
+ * uses for tensor-parallel inference (Section 2.1: allreduce aggregates the
+ * ranks' partial activations, allgather assembles every rank's chunk in every
+ * rank's buffer, reduce-scatter is named with them in Section 2.2), executed
+ * with the latency-optimised direct / all-pairs algorithm (Section 5.1), and
+ * the thread-block placement idea of Section 4.2 (Algorithm 1) mapped onto SMs.
+ *
+ * Numerics (bf16): dst = rne_bf16((((f(src[0]) + f(src[1])) + ...) + f(src[N-1])))
+ * with every partial sum an IEEE binary32 (round to nearest even, subnormals
+ * kept), ranks folded in the fixed order 0..N-1 starting from rank 0's value,
+ * and ONE final round-to-nearest-even to bf16.  A NaN result is the canonical
+ * 0x7FFF.  Every destination receives the same bits.  Allgather is a bit copy.
+ *
+ * Conventions, all entry points:
+ *  - `src` / `dst` are HOST arrays of `nranks` DEVICE pointers (except in
+ *    nuna_allreduce_host).  The arrays are read during the call and may be
+ *    freed on return.  The caller owns every rank buffer.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream);
+ *    collective calls are asynchronous on it and perform no host
+ *    synchronisation, no allocation and no host<->device copy once the
+ *    per-device context exists (see nuna_init), so they can be stream-captured.
+ *  - The return value is a nuna_status_t.  Argument errors launch nothing.
+ *    Conditions detected on the device (a barrier that timed out) are latched
+ *    in a status word read by nuna_device_status.
+ *  - 1 <= nranks <= NUNA_MAX_RANKS.  count == 0 returns NUNA_OK without a
+ *    launch.  Every pointer must be 16-byte aligned (NUNA_ERR_ALIGNMENT).
+ *    No destination range may overlap a source range or another destination
+ *    range (NUNA_ERR_ALIAS): in the emulation another rank's thread blocks
+ *    may still be reading a source, so in-place operation is not defined.
+ *  - Sizes quoted in KB/MB anywhere in this project are binary.
+ */
+#ifndef NUNA_H
+#define NUNA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    NUNA_OK = 0,
+    NUNA_ERR_INVALID_ARG = 1,
+    NUNA_ERR_UNSUPPORTED_DTYPE = 2,
+    NUNA_ERR_ALIGNMENT = 3,
+    NUNA_ERR_ALIAS = 4,
+    NUNA_ERR_CUDA = 5,
+    NUNA_ERR_TIMEOUT = 6,
+    NUNA_ERR_CAPTURING = 7,
+    NUNA_ERR_TOO_MANY_RANKS = 8,
+    NUNA_ERR_TOO_LARGE = 9
+} nuna_status_t;
+
+typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* only NUNA_BF16 is implemented */
+
+#define NUNA_MAX_RANKS 16
+
+/* `flags`, bits 0-1: thread-block placement (Section 4.2 / Section 5.3 baseline). */
+#define NUNA_PLACE_ROUNDROBIN 0u   /* locality-unaware: work item i -> thread block i mod grid          */
+#define NUNA_PLACE_AWARE      1u   /* persistent blocks pull the work planned for their SM's domain      */
+#define NUNA_PLACE_AUTO       2u   /* AWARE where the installed topology says it helps, else ROUNDROBIN  */
+#define NUNA_PLACE_MASK       3u
+/* `flags`, bit 4 (nuna_allreduce_twoshot only): the reducing block stores its tile straight into all N
+ * destinations, with no intermediate shard and no barrier.                                             */
+#define NUNA_TWOSHOT_PUT      16u
+
+/* Create the calling thread's current device's context (flag-barrier words, status word, work cursors,
+ * two-shot shard scratch of `scratch_bytes`).  Called implicitly by the first collective on a device;
+ * call it explicitly before stream capture, because it allocates.  Growing the scratch later also
+ * allocates.  Returns NUNA_ERR_CUDA if no device is usable.                                            */
+int nuna_init(size_t scratch_bytes);
+
+/* One-shot allreduce (Section 5.1, direct algorithm): every emulated rank d reads all N sources and
+ * writes dst[d].  src[r], dst[d]: `count` elements each.  Work item = (tile, destination rank).       */
+int nuna_allreduce_oneshot(const void* const* src, void* const* dst, int nranks,
+                           size_t count, int dtype, unsigned flags, void* stream);
+
+/* Two-shot allreduce: reduce-scatter over N contiguous chunks (emulated rank r reduces chunk r), an
+ * in-kernel flag barrier among the persistent thread blocks, then a put-style allgather of the chunks
+ * into every destination.  Same bits as the one-shot.  Any `count`; chunk = ceil(count/N) rounded up
+ * to 8 elements, trailing chunks may be short or empty.  Uses the context's shard scratch
+ * (count*elemsize bytes, grown on demand) unless NUNA_TWOSHOT_PUT is set.  Calls that share the
+ * context must be stream-ordered with respect to each other.                                          */
+int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
+                           size_t count, int dtype, unsigned flags, void* stream);
+
+/* Reduce-scatter: src[k] holds nranks*shard_count elements, dst[r] holds shard_count elements;
+ * dst[r][j] = fold over k of src[k][r*shard_count + j].                                               */
+int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks,
+                        size_t shard_count, int dtype, unsigned flags, void* stream);
+
+/* Allgather in the paper's form (Figure "Allocation_Diagram": local load, remote store): src[r] holds
+ * shard_count elements, every dst[d] holds nranks*shard_count; dst[d][r*shard_count + j] = src[r][j],
+ * copied bit for bit.                                                                                   */
+int nuna_allgather(const void* const* src, void* const* dst, int nranks,
+                   size_t shard_count, int dtype, unsigned flags, void* stream);
+
+/* End-to-end variant with HOST buffers: src[r] / dst[d] are HOST pointers to `count` elements (pinned
+ * or pageable).  Copies the sources to library-owned device staging buffers, runs the one-shot
+ * (two_shot == 0) or two-shot allreduce, copies every destination back and synchronises.  Allocates
+ * staging on first use or growth.                                                                       */
+int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks,
+                        size_t count, int dtype, unsigned flags, int two_shot);
+
+/* Reads and clears the device status word of the current device (NUNA_OK or NUNA_ERR_TIMEOUT) after
+ * synchronising the device.  After a timeout the barrier words are re-initialised.                     */
+int nuna_device_status(int* out);
+
+/* Number of kernels this library has launched on any device since load (the callers' launch count).   */
+unsigned long long nuna_launch_count(void);
+
+const char* nuna_status_string(int status);
+
+/* Frees the current device's context (scratch, staging, graphs are NOT freed: destroy chains first).  */
+int nuna_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NUNA_H */

@@ -1,0 +1,466 @@
+// Host side of the C ABI: argument checks, per-device context, launch configuration.
+#include "nuna_internal.h"
+
+#include <algorithm>
+#include <atomic>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <type_traits>
+
+namespace nuna {
+
+std::atomic<unsigned long long> g_launches{0};
+static std::mutex g_ctx_mutex;
+static Context* g_ctx[kMaxDevices] = {};
+
+static int env_int(const char* name, int fallback)
+{
+    const char* s = getenv(name);
+    return (s && *s) ? atoi(s) : fallback;
+}
+
+int init_barrier_words(Context* c)
+{
+    return cudaMemset(c->bw, 0, sizeof(BarrierWords)) == cudaSuccess ? NUNA_OK : NUNA_ERR_CUDA;
+}
+
+// Returns the current device's context, creating it on first use (allocates: not capturable).
+int get_context(Context** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return NUNA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_ctx_mutex);
+    if (!g_ctx[dev]) {
+        Context* c = new Context();
+        c->device = dev;
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { delete c; return NUNA_ERR_CUDA; }
+        c->num_sms = prop.multiProcessorCount;
+        c->l2_bytes = (size_t)prop.l2CacheSize;
+        if (cudaMalloc(&c->bw, sizeof(BarrierWords)) != cudaSuccess) { delete c; return NUNA_ERR_CUDA; }
+        if (init_barrier_words(c) != NUNA_OK) { cudaFree(c->bw); delete c; return NUNA_ERR_CUDA; }
+        c->timeout_ns = (unsigned long long)env_int("NUNA_TIMEOUT_MS", 1000) * 1000000ull;
+        c->blocks_override = env_int("NUNA_BLOCKS", 0);
+        c->unroll_override = env_int("NUNA_UNROLL", 0);
+        g_ctx[dev] = c;
+    }
+    *out = g_ctx[dev];
+    return NUNA_OK;
+}
+
+int ensure_scratch(Context* c, size_t bytes)
+{
+    if (bytes <= c->scratch_bytes) return NUNA_OK;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    (void)cs;
+    void* p = nullptr;
+    const size_t want = (bytes + 255) & ~(size_t)255;
+    if (cudaMalloc(&p, want) != cudaSuccess) return NUNA_ERR_CUDA;
+    if (c->scratch) cudaFree(c->scratch);
+    c->scratch = p;
+    c->scratch_bytes = want;
+    return NUNA_OK;
+}
+
+// ---- argument validation -------------------------------------------------------------------
+
+static bool overlaps(const void* a, size_t na, const void* b, size_t nb)
+{
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return na && nb && a0 < b0 + nb && b0 < a0 + na;
+}
+
+int check_args(const void* const* src, void* const* dst, int nranks, size_t src_elems, size_t dst_elems,
+               int dtype, unsigned flags, bool device_ptrs)
+{
+    if (nranks > NUNA_MAX_RANKS) return NUNA_ERR_TOO_MANY_RANKS;
+    if (nranks < 1) return NUNA_ERR_INVALID_ARG;
+    if (dtype != NUNA_BF16) return (dtype == NUNA_F16 || dtype == NUNA_F32) ? NUNA_ERR_UNSUPPORTED_DTYPE
+                                                                             : NUNA_ERR_UNSUPPORTED_DTYPE;
+    if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT)) != 0u || (flags & NUNA_PLACE_MASK) == 3u)
+        return NUNA_ERR_INVALID_ARG;
+    if (src_elems > ((size_t)1 << 40) || dst_elems > ((size_t)1 << 40)) return NUNA_ERR_TOO_LARGE;
+    if (src_elems == 0 && dst_elems == 0) return NUNA_OK;
+    if (!src || !dst) return NUNA_ERR_INVALID_ARG;
+    for (int r = 0; r < nranks; ++r) {
+        if (!src[r] || !dst[r]) return NUNA_ERR_INVALID_ARG;
+        if (device_ptrs && (((uintptr_t)src[r] | (uintptr_t)dst[r]) & 15u)) return NUNA_ERR_ALIGNMENT;
+    }
+    const size_t sb = src_elems * 2, db = dst_elems * 2;
+    for (int d = 0; d < nranks; ++d) {
+        for (int r = 0; r < nranks; ++r)
+            if (overlaps(dst[d], db, src[r], sb)) return NUNA_ERR_ALIAS;
+        for (int e = d + 1; e < nranks; ++e)
+            if (overlaps(dst[d], db, dst[e], db)) return NUNA_ERR_ALIAS;
+    }
+    return NUNA_OK;
+}
+
+static RankPtrs make_ptrs(const void* const* src, void* const* dst, int nranks)
+{
+    RankPtrs p;
+    memset(&p, 0, sizeof p);
+    for (int r = 0; r < nranks; ++r) {
+        p.src[r] = reinterpret_cast<const uint4*>(src[r]);
+        p.dst[r] = reinterpret_cast<uint4*>(dst[r]);
+    }
+    return p;
+}
+
+// ---- launch configuration --------------------------------------------------------------------
+
+// Vectors per thread per item.  Chosen so a thread keeps about 8-16 independent 16-byte loads in
+// flight whatever N is, without pushing register use past two or three blocks per SM.
+static int pick_unroll(const Context* c, int nranks)
+{
+    int u = nranks >= 8 ? 1 : nranks >= 4 ? 2 : 4;
+    if (c->unroll_override == 1 || c->unroll_override == 2 || c->unroll_override == 4) u = c->unroll_override;
+    while (u > 1 && u * nranks > 16) u >>= 1;
+    return u;
+}
+
+template <typename K>
+static int occupancy(Context* c, K kernel, int* cache)
+{
+    if (*cache == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, 0) != cudaSuccess || n < 1) n = 1;
+        *cache = n;
+    }
+    (void)c;
+    return *cache;
+}
+
+static unsigned pick_grid(const Context* c, size_t nitems, int blocks_per_sm)
+{
+    size_t cap = (size_t)c->num_sms * (size_t)blocks_per_sm;
+    if (c->blocks_override > 0) cap = (size_t)c->blocks_override;
+    return (unsigned)std::max<size_t>(1, std::min(nitems, cap));
+}
+
+template <typename... Args, typename... Act>
+static int launch(void (*kernel)(Args...), unsigned grid, cudaStream_t stream, bool cooperative, Act&&... args)
+{
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    int nattr = 0;
+    if (cooperative) {
+        attr[nattr].id = cudaLaunchAttributeCooperative;
+        attr[nattr].val.cooperative = 1;
+        ++nattr;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = nattr;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<Args>(args)...);
+    if (e != cudaSuccess) {
+        fprintf(stderr, "nuna: kernel launch failed: %s\n", cudaGetErrorString(e));
+        return NUNA_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return NUNA_OK;
+}
+
+// Compile-time dispatch over the rank count N and the unroll factor U (N * U <= 16 vectors in flight).
+template <int V> using IC = std::integral_constant<int, V>;
+
+template <int N, typename F>
+static int dispatch_u(int u, F&& f)
+{
+    if constexpr (N * 4 <= 16) { if (u == 4) return f(IC<N>{}, IC<4>{}); }
+    if constexpr (N * 2 <= 16) { if (u >= 2) return f(IC<N>{}, IC<2>{}); }
+    return f(IC<N>{}, IC<1>{});
+}
+
+template <typename F>
+static int dispatch(int nranks, int u, F&& f)
+{
+    switch (nranks) {
+        case 1: return dispatch_u<1>(u, f);   case 2: return dispatch_u<2>(u, f);
+        case 3: return dispatch_u<3>(u, f);   case 4: return dispatch_u<4>(u, f);
+        case 5: return dispatch_u<5>(u, f);   case 6: return dispatch_u<6>(u, f);
+        case 7: return dispatch_u<7>(u, f);   case 8: return dispatch_u<8>(u, f);
+        case 9: return dispatch_u<9>(u, f);   case 10: return dispatch_u<10>(u, f);
+        case 11: return dispatch_u<11>(u, f); case 12: return dispatch_u<12>(u, f);
+        case 13: return dispatch_u<13>(u, f); case 14: return dispatch_u<14>(u, f);
+        case 15: return dispatch_u<15>(u, f); case 16: return dispatch_u<16>(u, f);
+        default: return NUNA_ERR_TOO_MANY_RANKS;
+    }
+}
+#define NUNA_NU(n_, u_) constexpr int N = decltype(n_)::value; constexpr int U = decltype(u_)::value; (void)U
+
+static size_t ceil_div(size_t a, size_t b) { return (a + b - 1) / b; }
+
+// ---- collectives ---------------------------------------------------------------------------------
+
+int launch_oneshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream)
+{
+    (void)flags;
+    const size_t nvec = count / kVecElems;
+    return dispatch(nranks, pick_unroll(c, nranks), [&](auto n_, auto u_) -> int {
+        NUNA_NU(n_, u_);
+        static int occ = 0;
+        auto k = k_oneshot_rr<N, U>;
+        const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
+        const size_t nitems = std::max<size_t>(ntiles * N, (count % kVecElems) ? (size_t)N : 0);
+        const unsigned grid = pick_grid(c, nitems, occupancy(c, k, &occ));
+        return launch(k, grid, stream, false, p, count, ntiles);
+    });
+}
+
+int launch_twoshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream)
+{
+    const size_t nvec = count / kVecElems;
+    if (flags & NUNA_TWOSHOT_PUT) {
+        return dispatch(nranks, pick_unroll(c, nranks), [&](auto n_, auto u_) -> int {
+            NUNA_NU(n_, u_);
+            static int occ = 0;
+            auto k = k_twoshot_put<N, U>;
+            const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
+            const unsigned grid = pick_grid(c, std::max<size_t>(ntiles, 1), occupancy(c, k, &occ));
+            return launch(k, grid, stream, false, p, count, ntiles);
+        });
+    }
+    // chunk = ceil(count / N) rounded up to whole vectors
+    const size_t chunk_vec = ceil_div(ceil_div(count, (size_t)nranks), (size_t)kVecElems);
+    return dispatch(nranks, pick_unroll(c, nranks), [&](auto n_, auto u_) -> int {
+        NUNA_NU(n_, u_);
+        static int occ = 0;
+        auto k = k_twoshot_fused<N, U>;
+        const size_t tiles_per_chunk = ceil_div(chunk_vec, (size_t)kThreads * U);
+        // every block must be resident for the flag barrier: never more than the device holds at once
+        size_t cap = (size_t)c->num_sms * (size_t)occupancy(c, k, &occ);
+        if (c->blocks_override > 0) cap = std::min<size_t>(cap, (size_t)c->blocks_override);
+        const unsigned grid = (unsigned)std::max<size_t>(1, std::min(tiles_per_chunk * N, cap));
+        return launch(k, grid, stream, true, p, reinterpret_cast<uint4*>(c->scratch), count, chunk_vec,
+                      c->bw, c->timeout_ns);
+    });
+}
+
+int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shard, cudaStream_t stream)
+{
+    if (shard % kVecElems) {
+        const unsigned grid = pick_grid(c, ceil_div(shard * nranks, kThreads), 8);
+        return dispatch(nranks, 1, [&](auto n_, auto u_) -> int {
+            NUNA_NU(n_, u_);
+            return launch(k_reduce_scatter_scalar<N>, grid, stream, false, p, shard);
+        });
+    }
+    const size_t shard_vec = shard / kVecElems;
+    return dispatch(nranks, pick_unroll(c, nranks), [&](auto n_, auto u_) -> int {
+        NUNA_NU(n_, u_);
+        static int occ = 0;
+        auto k = k_reduce_scatter<N, U>;
+        const size_t tiles = ceil_div(shard_vec, (size_t)kThreads * U);
+        const unsigned grid = pick_grid(c, tiles * N, occupancy(c, k, &occ));
+        return launch(k, grid, stream, false, p, shard_vec, tiles);
+    });
+}
+
+int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, cudaStream_t stream)
+{
+    if (shard % kVecElems) {
+        const unsigned grid = pick_grid(c, ceil_div(shard * nranks, kThreads), 8);
+        return launch(k_allgather_scalar, grid, stream, false, p, nranks, shard);
+    }
+    const size_t shard_vec = shard / kVecElems;
+    static int occ = 0;
+    constexpr int U = 2;
+    auto k = k_allgather<U>;
+    const size_t tiles = ceil_div(shard_vec, (size_t)kThreads * U);
+    const unsigned grid = pick_grid(c, tiles * nranks, occupancy(c, k, &occ));
+    return launch(k, grid, stream, false, p, nranks, shard_vec, tiles);
+}
+
+}  // namespace nuna
+
+using namespace nuna;
+
+extern "C" {
+
+int nuna_init(size_t scratch_bytes)
+{
+    Context* c = nullptr;
+    int st = get_context(&c);
+    if (st != NUNA_OK) return st;
+    std::lock_guard<std::mutex> lock(c->mutex);
+    return ensure_scratch(c, scratch_bytes);
+}
+
+int nuna_allreduce_oneshot(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
+                           unsigned flags, void* stream)
+{
+    int st = check_args(src, dst, nranks, count, count, dtype, flags & ~NUNA_TWOSHOT_PUT, true);
+    if (st != NUNA_OK || count == 0) return st;
+    if (flags & NUNA_TWOSHOT_PUT) return NUNA_ERR_INVALID_ARG;
+    Context* c = nullptr;
+    if ((st = get_context(&c)) != NUNA_OK) return st;
+    return launch_oneshot(c, make_ptrs(src, dst, nranks), nranks, count, flags, (cudaStream_t)stream);
+}
+
+int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
+                           unsigned flags, void* stream)
+{
+    int st = check_args(src, dst, nranks, count, count, dtype, flags, true);
+    if (st != NUNA_OK || count == 0) return st;
+    Context* c = nullptr;
+    if ((st = get_context(&c)) != NUNA_OK) return st;
+    if (!(flags & NUNA_TWOSHOT_PUT)) {
+        std::lock_guard<std::mutex> lock(c->mutex);
+        const size_t need = (count * 2 + 15) & ~(size_t)15;
+        if (need > c->scratch_bytes) {
+            cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+            if (cudaStreamIsCapturing((cudaStream_t)stream, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone)
+                return NUNA_ERR_CAPTURING;             // growing the scratch allocates: call nuna_init first
+            if ((st = ensure_scratch(c, need)) != NUNA_OK) return st;
+        }
+    }
+    return launch_twoshot(c, make_ptrs(src, dst, nranks), nranks, count, flags, (cudaStream_t)stream);
+}
+
+int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks, size_t shard_count, int dtype,
+                        unsigned flags, void* stream)
+{
+    if (nranks >= 1 && nranks <= NUNA_MAX_RANKS && shard_count > ((size_t)1 << 40) / (size_t)nranks)
+        return NUNA_ERR_TOO_LARGE;
+    int st = check_args(src, dst, nranks, shard_count * (size_t)(nranks > 0 ? nranks : 0), shard_count, dtype,
+                        flags & ~NUNA_TWOSHOT_PUT, true);
+    if (st != NUNA_OK || shard_count == 0) return st;
+    if (flags & NUNA_TWOSHOT_PUT) return NUNA_ERR_INVALID_ARG;
+    Context* c = nullptr;
+    if ((st = get_context(&c)) != NUNA_OK) return st;
+    return launch_reduce_scatter(c, make_ptrs(src, dst, nranks), nranks, shard_count, (cudaStream_t)stream);
+}
+
+int nuna_allgather(const void* const* src, void* const* dst, int nranks, size_t shard_count, int dtype,
+                   unsigned flags, void* stream)
+{
+    if (nranks >= 1 && nranks <= NUNA_MAX_RANKS && shard_count > ((size_t)1 << 40) / (size_t)nranks)
+        return NUNA_ERR_TOO_LARGE;
+    int st = check_args(src, dst, nranks, shard_count, shard_count * (size_t)(nranks > 0 ? nranks : 0), dtype,
+                        flags & ~NUNA_TWOSHOT_PUT, true);
+    if (st != NUNA_OK || shard_count == 0) return st;
+    if (flags & NUNA_TWOSHOT_PUT) return NUNA_ERR_INVALID_ARG;
+    Context* c = nullptr;
+    if ((st = get_context(&c)) != NUNA_OK) return st;
+    return launch_allgather(c, make_ptrs(src, dst, nranks), nranks, shard_count, (cudaStream_t)stream);
+}
+
+int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
+                        unsigned flags, int two_shot)
+{
+    int st = check_args(src, dst, nranks, count, count, dtype, flags, false);
+    if (st != NUNA_OK || count == 0) return st;
+    if (!two_shot && (flags & NUNA_TWOSHOT_PUT)) return NUNA_ERR_INVALID_ARG;
+    Context* c = nullptr;
+    if ((st = get_context(&c)) != NUNA_OK) return st;
+    std::lock_guard<std::mutex> lock(c->mutex);
+    const size_t bytes = count * 2;
+    const size_t slot = (bytes + 255) & ~(size_t)255;
+    const size_t need = slot * 2 * (size_t)nranks;
+    if (need > c->staging_bytes) {
+        if (c->staging) cudaFree(c->staging);
+        c->staging = nullptr;
+        c->staging_bytes = 0;
+        if (cudaMalloc(&c->staging, need) != cudaSuccess) return NUNA_ERR_CUDA;
+        c->staging_bytes = need;
+    }
+    if (!c->stream && cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking) != cudaSuccess) return NUNA_ERR_CUDA;
+    if (two_shot && !(flags & NUNA_TWOSHOT_PUT) && (st = ensure_scratch(c, slot)) != NUNA_OK) return st;
+    const void* dsrc[NUNA_MAX_RANKS];
+    void* ddst[NUNA_MAX_RANKS];
+    char* base = static_cast<char*>(c->staging);
+    for (int r = 0; r < nranks; ++r) {
+        dsrc[r] = base + slot * (size_t)r;
+        ddst[r] = base + slot * (size_t)(nranks + r);
+        if (cudaMemcpyAsync(const_cast<void*>(dsrc[r]), src[r], bytes, cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+            return NUNA_ERR_CUDA;
+    }
+    const RankPtrs p = make_ptrs(dsrc, ddst, nranks);
+    st = two_shot ? launch_twoshot(c, p, nranks, count, flags, c->stream)
+                  : launch_oneshot(c, p, nranks, count, flags, c->stream);
+    if (st != NUNA_OK) return st;
+    for (int d = 0; d < nranks; ++d)
+        if (cudaMemcpyAsync(dst[d], ddst[d], bytes, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
+            return NUNA_ERR_CUDA;
+    return cudaStreamSynchronize(c->stream) == cudaSuccess ? NUNA_OK : NUNA_ERR_CUDA;
+}
+
+int nuna_device_status(int* out)
+{
+    if (!out) return NUNA_ERR_INVALID_ARG;
+    Context* c = nullptr;
+    int st = get_context(&c);
+    if (st != NUNA_OK) return st;
+    if (cudaDeviceSynchronize() != cudaSuccess) return NUNA_ERR_CUDA;
+    BarrierWords h;
+    if (cudaMemcpy(&h, c->bw, sizeof h, cudaMemcpyDeviceToHost) != cudaSuccess) return NUNA_ERR_CUDA;
+    *out = (int)h.status;
+    if (h.status != 0) return init_barrier_words(c);
+    return NUNA_OK;
+}
+
+unsigned long long nuna_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* nuna_status_string(int status)
+{
+    switch (status) {
+        case NUNA_OK: return "ok";
+        case NUNA_ERR_INVALID_ARG: return "invalid argument";
+        case NUNA_ERR_UNSUPPORTED_DTYPE: return "unsupported dtype";
+        case NUNA_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case NUNA_ERR_ALIAS: return "destination overlaps a source or another destination";
+        case NUNA_ERR_CUDA: return "CUDA runtime error";
+        case NUNA_ERR_TIMEOUT: return "flag barrier timed out";
+        case NUNA_ERR_CAPTURING: return "operation would allocate or synchronise during stream capture";
+        case NUNA_ERR_TOO_MANY_RANKS: return "more than NUNA_MAX_RANKS ranks";
+        case NUNA_ERR_TOO_LARGE: return "size beyond the supported maximum";
+        default: return "unknown status";
+    }
+}
+
+int nuna_shutdown(void)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return NUNA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_ctx_mutex);
+    Context* c = g_ctx[dev];
+    if (!c) return NUNA_OK;
+    cudaDeviceSynchronize();
+    if (c->bw) cudaFree(c->bw);
+    if (c->scratch) cudaFree(c->scratch);
+    if (c->staging) cudaFree(c->staging);
+    if (c->stream) cudaStreamDestroy(c->stream);
+    delete c;
+    g_ctx[dev] = nullptr;
+    return NUNA_OK;
+}
+
+/* Test hook (not part of the public header): every block of a `grid`-block launch arrives at a flag
+ * barrier that expects `expected` arrivals and waits at most timeout_ms.  Writes how many blocks
+ * passed.  With expected > grid nothing ever completes the barrier, the waits run out, and the
+ * status word latches NUNA_ERR_TIMEOUT -- without trapping or hanging the device.                    */
+int nuna_debug_barrier_selftest(unsigned grid, unsigned expected, unsigned timeout_ms, unsigned* passed)
+{
+    Context* c = nullptr;
+    int st = get_context(&c);
+    if (st != NUNA_OK) return st;
+    if (!passed || grid == 0 || grid > (unsigned)c->num_sms || expected == 0) return NUNA_ERR_INVALID_ARG;
+    unsigned* d = nullptr;
+    if (cudaMalloc(&d, sizeof(unsigned)) != cudaSuccess) return NUNA_ERR_CUDA;
+    cudaMemset(d, 0, sizeof(unsigned));
+    st = launch(k_barrier_selftest, grid, (cudaStream_t)0, true, c->bw, expected,
+                (unsigned long long)timeout_ms * 1000000ull, d);
+    if (st == NUNA_OK && cudaDeviceSynchronize() != cudaSuccess) st = NUNA_ERR_CUDA;
+    if (st == NUNA_OK && cudaMemcpy(passed, d, sizeof(unsigned), cudaMemcpyDeviceToHost) != cudaSuccess) st = NUNA_ERR_CUDA;
+    cudaFree(d);
+    return st;
+}
+
+}  // extern "C"

@@ -1,0 +1,42 @@
+// Shared by the library's own translation units (never by the oracle).
+#pragma once
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <mutex>
+
+#include "../../include/nuna.h"
+#include "nuna_kernels.cuh"
+
+namespace nuna {
+
+constexpr int kMaxDevices = 64;
+
+struct Context {
+    int device = -1;
+    int num_sms = 0;
+    size_t l2_bytes = 0;
+    BarrierWords* bw = nullptr;          // flag-barrier words + latched status, device memory
+    void* scratch = nullptr;             // two-shot shard intermediate
+    size_t scratch_bytes = 0;
+    void* staging = nullptr;             // device copies of host buffers (nuna_allreduce_host)
+    size_t staging_bytes = 0;
+    cudaStream_t stream = nullptr;       // private stream of the host-buffer entry point
+    unsigned long long timeout_ns = 1000000000ull;
+    int blocks_override = 0;             // NUNA_BLOCKS
+    int unroll_override = 0;             // NUNA_UNROLL
+    std::mutex mutex;
+};
+
+extern std::atomic<unsigned long long> g_launches;
+
+int get_context(Context** out);
+int ensure_scratch(Context* c, size_t bytes);
+int check_args(const void* const* src, void* const* dst, int nranks, size_t src_elems, size_t dst_elems,
+               int dtype, unsigned flags, bool device_ptrs);
+int launch_oneshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream);
+int launch_twoshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream);
+int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shard, cudaStream_t stream);
+int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, cudaStream_t stream);
+
+}  // namespace nuna

@@ -1,0 +1,252 @@
+"""Parity of the CUDA library against the CPU oracle, through the C ABI.  Bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_00867_b200 import binding as nb
+from paper_2608_00867_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+GUARD = 64          # sentinel elements on each side of every destination
+SENTINEL = 0x5A5A
+POISON = 0xDEAD
+
+
+def upload(arrs):
+    return [torch.from_numpy(a.view(np.int16).copy()).cuda() for a in arrs]
+
+
+class Dst:
+    """Destination buffers with guard zones; the payload starts 16-byte aligned."""
+
+    def __init__(self, n, count):
+        self.count = count
+        self.full = []
+        self.view = []
+        for _ in range(n):
+            t = torch.full((count + 2 * GUARD,), SENTINEL, dtype=torch.int16, device="cuda")
+            t[GUARD:GUARD + count] = np.int16(np.uint16(POISON).view(np.int16))
+            self.full.append(t)
+            self.view.append(t[GUARD:GUARD + count])
+
+    def numpy(self):
+        torch.cuda.synchronize()
+        out = []
+        for t in self.full:
+            h = t.cpu().numpy().view(np.uint16)
+            assert (h[:GUARD] == SENTINEL).all() and (h[GUARD + self.count:] == SENTINEL).all(), "guard zone overwritten"
+            out.append(h[GUARD:GUARD + self.count].copy())
+        return out
+
+
+def is_nan(a):
+    return ((a & 0x7F80) == 0x7F80) & ((a & 0x007F) != 0)
+
+
+def assert_same_bits(got, want, what=""):
+    """Equal bit patterns; where the oracle has a NaN the GPU must have a NaN (payload unpinned)."""
+    assert got.shape == want.shape, what
+    nan = is_nan(want)
+    assert np.array_equal(is_nan(got), nan), what + ": NaN positions differ"
+    bad = np.nonzero((got != want) & ~nan)[0]
+    assert bad.size == 0, f"{what}: {bad.size} mismatches, first at {bad[:5]}: got {got[bad[:5]]} want {want[bad[:5]]}"
+
+
+COUNTS = [1, 7, 8, 9, 15, 16, 17, 2047, 2048, 2049, 4096, 6151, 100003, 262144]
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16])
+@pytest.mark.parametrize("algo", ["oneshot", "twoshot", "twoshot_put"])
+def test_allreduce_special_values_all_counts(n, algo):
+    for count in COUNTS:
+        src = workloads.special_values(n, count, seed=1000 * n + count % 997)
+        want = oracle.allreduce(src, nthreads=4)
+        dsrc, dst = upload(src), Dst(n, count)
+        if algo == "oneshot":
+            nb.nuna_allreduce_oneshot(dsrc, dst.view, count)
+        else:
+            nb.nuna_allreduce_twoshot(dsrc, dst.view, count, flags=nb.NUNA_TWOSHOT_PUT if algo == "twoshot_put" else 0)
+        got = dst.numpy()
+        for d in range(n):
+            assert_same_bits(got[d], want[d], f"{algo} n={n} count={count} dst={d}")
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
+def test_config_small_two_ranks():
+    w = workloads.config_small_oneshot()
+    src = workloads.make(w)
+    want = oracle.allreduce(src)
+    dst = Dst(w.nranks, w.count)
+    nb.nuna_allreduce_oneshot(upload(src), dst.view, w.count)
+    got = dst.numpy()
+    for d in range(w.nranks):
+        assert np.array_equal(got[d], want[d])
+
+
+@pytest.mark.parametrize("flags", [nb.NUNA_PLACE_ROUNDROBIN, nb.NUNA_PLACE_AWARE, nb.NUNA_PLACE_AUTO])
+def test_config_decode_activation_all_placements(flags):
+    w = workloads.config_decode_activation()
+    src = workloads.make(w)
+    want = oracle.allreduce(src, nthreads=4)
+    dsrc = upload(src)
+    for call in (nb.nuna_allreduce_oneshot, nb.nuna_allreduce_twoshot):
+        dst = Dst(w.nranks, w.count)
+        call(dsrc, dst.view, w.count, flags=flags)
+        got = dst.numpy()
+        for d in range(w.nranks):
+            assert np.array_equal(got[d], want[d])
+
+
+@pytest.mark.parametrize("n,shard", [(8, 4096), (8, 1000), (16, 33), (3, 8), (5, 2049), (8, 65536), (2, 1)])
+def test_reduce_scatter_and_allgather(n, shard):
+    src = workloads.special_values(n, n * shard, seed=n * 31 + shard)
+    want_rs = oracle.reduce_scatter(src, nthreads=4)
+    dsrc = upload(src)
+    rs = Dst(n, shard)
+    nb.nuna_reduce_scatter(dsrc, rs.view, shard)
+    got_rs = rs.numpy()
+    for r in range(n):
+        assert_same_bits(got_rs[r], want_rs[r], f"rs n={n} shard={shard} r={r}")
+    # allgather of the GPU's own shards: raw bit copy, NaN payloads included
+    want_ag = oracle.allgather(got_rs)
+    ag = Dst(n, n * shard)
+    nb.nuna_allgather(rs.view, ag.view, shard)
+    got_ag = ag.numpy()
+    for d in range(n):
+        assert np.array_equal(got_ag[d], want_ag[d])
+    # allreduce == allgather(reduce_scatter) byte for byte (NaN payload aside)
+    ar = Dst(n, n * shard)
+    nb.nuna_allreduce_oneshot(dsrc, ar.view, n * shard)
+    got_ar = ar.numpy()
+    for d in range(n):
+        assert_same_bits(got_ag[d], got_ar[d], "ar vs ag(rs)")
+
+
+def test_config_allgather16_raw_bits():
+    w = workloads.config_allgather16()
+    rng = np.random.Generator(np.random.PCG64(w.seed))
+    for src in (workloads.make(w),
+                [rng.integers(0, 1 << 16, size=w.count, dtype=np.uint32).astype(np.uint16) for _ in range(w.nranks)]):
+        want = oracle.allgather(src)
+        dst = Dst(w.nranks, w.nranks * w.count)
+        nb.nuna_allgather(upload(src), dst.view, w.count)
+        got = dst.numpy()
+        for d in range(w.nranks):
+            assert np.array_equal(got[d], want[d])
+
+
+def test_sweep_sizes_one_and_two_shot_agree_with_oracle():
+    for w in workloads.config_size_sweep(13, 22):
+        src = workloads.make(w)
+        want = oracle.allreduce(src, nthreads=8)[0]
+        dsrc = upload(src)
+        for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_twoshot, 0),
+                            (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
+            dst = Dst(w.nranks, w.count)
+            call(dsrc, dst.view, w.count, flags=flags)
+            got = dst.numpy()
+            for d in range(w.nranks):
+                assert np.array_equal(got[d], want), (w.name, call.__name__, flags, d)
+
+
+def test_full_size_64MiB_sampled_columns_and_invariants():
+    """BASELINE's largest point, in the launch configuration the benchmark times."""
+    w = workloads.config_size_sweep(26, 26)[0]
+    n, count = w.nranks, w.count
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed)
+    dsrc = [torch.randn(count, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16).view(torch.int16)
+            for _ in range(n)]
+    # one "awkward" column block: wide exponent spread so the fold order is observable
+    sp = workloads.special_values(n, 4096, seed=5)
+    for r in range(n):
+        dsrc[r][count - 4096:] = torch.from_numpy(sp[r].view(np.int16)).cuda()
+    rng = np.random.Generator(np.random.PCG64(99))
+    idx = np.unique(np.concatenate([rng.integers(0, count, size=20000), np.arange(0, 4096),
+                                    np.arange(count - 6000, count), np.arange(count // 8 - 2048, count // 8 + 2048)]))
+    tidx = torch.from_numpy(idx).cuda()
+    cols = np.stack([t[tidx].cpu().numpy().view(np.uint16) for t in dsrc])          # [n, len(idx)]
+    want = oracle.allreduce([np.ascontiguousarray(c) for c in cols], nthreads=4)[0]
+    results = []
+    for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_twoshot, 0),
+                        (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
+        dst = [torch.full((count,), -1, dtype=torch.int16, device="cuda") for _ in range(n)]
+        call(dsrc, dst, count, flags=flags)
+        torch.cuda.synchronize()
+        assert_same_bits(dst[0][tidx].cpu().numpy().view(np.uint16), want, call.__name__)
+        for d in range(1, n):
+            assert torch.equal(dst[0], dst[d])                        # all destinations identical
+        results.append(dst[0].clone())
+        del dst
+    assert torch.equal(results[0], results[1]) and torch.equal(results[0], results[2])
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
+def test_graph_replay_gives_same_bits():
+    w = workloads.config_decode_activation()
+    src = workloads.make(w)
+    want = oracle.allreduce(src, nthreads=4)[0]
+    dsrc = upload(src)
+    dst = [torch.zeros(w.count, dtype=torch.int16, device="cuda") for _ in range(w.nranks)]
+    nb.nuna_init(2 * w.count)
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            nb.nuna_allreduce_oneshot(dsrc, dst, w.count, stream=s)
+            nb.nuna_allreduce_twoshot(dsrc, dst, w.count, stream=s)
+    for _ in range(3):
+        for t in dst:
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for t in dst:
+            assert np.array_equal(t.cpu().numpy().view(np.uint16), want)
+
+
+def test_host_buffer_entry_point():
+    for n, count, two in ((8, 32 * 8192, False), (8, 32 * 8192, True), (3, 1001, False), (3, 1001, True)):
+        src = workloads.rank_buffers(n, count, "normal", seed=77)
+        want = oracle.allreduce(src)[0]
+        dst = [np.zeros(count, dtype=np.uint16) for _ in range(n)]
+        nb.nuna_allreduce_host(src, dst, count, two_shot=two)
+        for d in range(n):
+            assert np.array_equal(dst[d], want)
+
+
+def test_argument_errors_launch_nothing():
+    a = [torch.zeros(64, dtype=torch.int16, device="cuda") for _ in range(2)]
+    b = [torch.zeros(64, dtype=torch.int16, device="cuda") for _ in range(2)]
+    before = nb.nuna_launch_count()
+    assert nb.nuna_allreduce_oneshot(a, b, 0) == nb.NUNA_OK
+    assert nb.nuna_allreduce_oneshot(a, a, 64, check=False) == nb.NUNA_ERR_ALIAS
+    assert nb.nuna_allreduce_oneshot(a, [b[0], b[0]], 64, check=False) == nb.NUNA_ERR_ALIAS
+    assert nb.nuna_allreduce_oneshot(a, [b[0], a[1][32:]], 32, check=False) == nb.NUNA_ERR_ALIAS
+    assert nb.nuna_allreduce_oneshot(a, [b[0], b[1][1:]], 8, check=False) == nb.NUNA_ERR_ALIGNMENT
+    assert nb.nuna_allreduce_oneshot(a, b, 64, dtype=nb.NUNA_F32, check=False) == nb.NUNA_ERR_UNSUPPORTED_DTYPE
+    assert nb.nuna_allreduce_oneshot(a, b, 64, flags=3, check=False) == nb.NUNA_ERR_INVALID_ARG
+    assert nb.nuna_allreduce_oneshot(a, b, 64, flags=nb.NUNA_TWOSHOT_PUT, check=False) == nb.NUNA_ERR_INVALID_ARG
+    assert nb.nuna_allreduce_oneshot(a * 9, b * 9, 64, check=False) == nb.NUNA_ERR_TOO_MANY_RANKS
+    assert nb.nuna_allreduce_oneshot([a[0], 0], b, 64, check=False) == nb.NUNA_ERR_INVALID_ARG
+    assert nb.nuna_launch_count() == before
+    with pytest.raises(nb.NunaError):
+        nb.nuna_allreduce_oneshot(a, a, 64)
+
+
+def test_flag_barrier_completes_and_times_out_cleanly():
+    st, passed = nb.debug_barrier_selftest(64, 64, 1000)
+    assert st == nb.NUNA_OK and passed == 64
+    assert nb.nuna_device_status() == nb.NUNA_OK
+    # a barrier nothing can complete: every wait runs out, the status word latches, nothing hangs
+    st, passed = nb.debug_barrier_selftest(32, 33, 50)
+    assert st == nb.NUNA_OK and passed == 0
+    assert nb.nuna_device_status() == nb.NUNA_ERR_TIMEOUT
+    assert nb.nuna_device_status() == nb.NUNA_OK            # cleared and barrier words re-initialised
+    # the context is still usable
+    w = workloads.config_decode_activation()
+    src = workloads.make(w)
+    dst = Dst(w.nranks, w.count)
+    nb.nuna_allreduce_twoshot(upload(src), dst.view, w.count)
+    assert np.array_equal(dst.numpy()[3], oracle.allreduce(src, nthreads=4)[0])
