@@ -112,6 +112,10 @@ int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks,
  * synchronising the device.  After a timeout the barrier words are re-initialised.                     */
 int nuna_device_status(int* out);
 
+/* Launches an empty kernel of `blocks` thread blocks with the collectives' block shape on `stream`: the
+ * single-kernel-launch floor that small-message latencies are reported against.                        */
+int nuna_launch_floor(unsigned blocks, void* stream);
+
 /* Number of kernels this library has launched on any device since load (the callers' launch count).   */
 unsigned long long nuna_launch_count(void);
 

@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
         L.nuna_init.restype = ctypes.c_int
         L.nuna_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
         L.nuna_device_status.restype = ctypes.c_int
+        L.nuna_launch_floor.argtypes = [ctypes.c_uint, ctypes.c_void_p]
+        L.nuna_launch_floor.restype = ctypes.c_int
         L.nuna_launch_count.argtypes = []
         L.nuna_launch_count.restype = ctypes.c_ulonglong
         L.nuna_status_string.argtypes = [ctypes.c_int]
@@ -136,6 +138,10 @@ def nuna_device_status() -> int:
     if st != NUNA_OK:
         raise NunaError(st, "nuna_device_status")
     return out.value
+
+
+def nuna_launch_floor(blocks: int, stream=None, check: bool = True) -> int:
+    return _finish(lib().nuna_launch_floor(blocks, _stream(stream)), "nuna_launch_floor", check)
 
 
 def nuna_launch_count() -> int:

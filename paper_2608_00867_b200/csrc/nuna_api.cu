@@ -406,6 +406,12 @@ int nuna_device_status(int* out)
     return NUNA_OK;
 }
 
+int nuna_launch_floor(unsigned blocks, void* stream)
+{
+    if (blocks == 0 || blocks > (1u << 20)) return NUNA_ERR_INVALID_ARG;
+    return launch(k_empty, blocks, (cudaStream_t)stream, false, 0);
+}
+
 unsigned long long nuna_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* nuna_status_string(int status)
