@@ -262,6 +262,7 @@ def run_gpu(args):
     # launch floor: the same graph shape with an empty kernel of the same grid
     grid_blocks = min(N_RANKS * -(-(count // 8) // 256), num_sms * 5)
     floor_us = per_call_us(lambda s, d, st: nb.nuna_launch_floor(grid_blocks, stream=st), sets, 1000, 3)
+    floor_pdl_us = per_call_us(lambda s, d, st: nb.nuna_launch_floor(grid_blocks, flags=nb.NUNA_LAUNCH_PDL, stream=st), sets, 1000, 3)
 
     extras = {}
     if True:
@@ -284,6 +285,7 @@ def run_gpu(args):
         # ---- message-size sweep, 8 ranks, 8 KiB .. 64 MiB per rank --------------------------------------
         algos = {
             "oneshot": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, stream=st)),
+            "oneshot_aware": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=nb.NUNA_PLACE_AWARE, stream=st)),
             "twoshot": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, stream=st)),
             "twoshot_put": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, flags=nb.NUNA_TWOSHOT_PUT, stream=st)),
         }
@@ -317,15 +319,37 @@ def run_gpu(args):
         torch.cuda.empty_cache()
 
         # ---- decode-step chain: 160 back-to-back one-shot allreduces in one graph ------------------------
+        # Two alternating source sets (attention-out / MLP-out partials), L2-resident as in decode.
+        variants = {
+            "roundrobin": nb.NUNA_PLACE_ROUNDROBIN,
+            "roundrobin_pdl": nb.NUNA_PLACE_ROUNDROBIN | nb.NUNA_LAUNCH_PDL,
+            "aware_pdl": nb.NUNA_PLACE_AWARE | nb.NUNA_LAUNCH_PDL,
+            "auto_resident_pdl": nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT | nb.NUNA_LAUNCH_PDL,
+        }
         for tokens in workloads.CHAIN_TOKENS:
             wc = workloads.config_decode_chain(tokens)
-            csets = make_sets(N_RANKS, wc.count, wc.count, 0, "normal", wc.seed, max_sets=2)   # attention-out / MLP-out
-            fn = lambda s, d, st, c=wc.count: nb.nuna_allreduce_oneshot(s, d, c, flags=nb.NUNA_PLACE_AUTO, stream=st)
-            g = capture(fn, csets, workloads.CHAIN_NODES)
-            ms = time_graph(g, 20, warm_replays=3)
-            chain_rows.append({"tokens": tokens, "bytes_per_rank": wc.bytes_per_rank, "nodes": workloads.CHAIN_NODES,
-                               "step_us": round(ms * 1e3 / 20, 2), "per_node_us": round(ms * 1e3 / 20 / workloads.CHAIN_NODES, 3)})
-            del g, csets
+            csets = make_sets(N_RANKS, wc.count, wc.count, 0, "normal", wc.seed, max_sets=2)
+            row = {"tokens": tokens, "bytes_per_rank": wc.bytes_per_rank, "nodes": workloads.CHAIN_NODES}
+            for vname, vflags in variants.items():
+                chain = nb.nuna_chain_create([c[0] for c in csets], [c[1] for c in csets], workloads.CHAIN_NODES,
+                                             wc.count, flags=vflags)
+                with torch.cuda.stream(stream):
+                    for _ in range(3):
+                        nb.nuna_chain_launch(chain, stream=stream)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    barrier()
+                    t0 = time.time()
+                    e0.record(stream)
+                    for _ in range(20):
+                        nb.nuna_chain_launch(chain, stream=stream)
+                    e1.record(stream)
+                    barrier()
+                    sampler.mark(t0, time.time())
+                ms = max_over_ranks(e0.elapsed_time(e1))
+                nb.nuna_chain_destroy(chain)
+                row[vname] = {"step_us": round(ms * 1e3 / 20, 2), "per_node_us": round(ms * 1e3 / 20 / workloads.CHAIN_NODES, 3)}
+            chain_rows.append(row)
+            del csets
 
     # ---- CPU baseline: the oracle as it stands, on this machine's cores (rank 0 at N = 1 only) -----------------
     cpu = None
@@ -366,7 +390,7 @@ def run_gpu(args):
                      "traffic": traffic, "peak_source": peak_src,
                      "note": "512 KiB per rank moves 8 MiB: 1.28 us at peak, so this size is latency-bound; "
                              "see sweep[] for the bandwidth-bound sizes",
-                     "launch_floor_us": round(floor_us, 3)},
+                     "launch_floor_us": round(floor_us, 3), "launch_floor_pdl_us": round(floor_pdl_us, 3)},
         "gpu_launches": K,
         "launches_since_load": int(launches_total),
         "device_status": status,

@@ -69,6 +69,16 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* on
 /* `flags`, bit 4 (nuna_allreduce_twoshot only): the reducing block stores its tile straight into all N
  * destinations, with no intermediate shard and no barrier.                                             */
 #define NUNA_TWOSHOT_PUT      16u
+/* `flags`, bit 5: hint that the sources were just written and are L2-resident (the decode case: a GEMM
+ * epilogue produced them).  NUNA_PLACE_AUTO uses the placement-aware kernel only under this hint, from
+ * 64 KiB per rank, and while 4 * nranks * bytes-per-rank fits in L2: the range where it was measured
+ * to be at least as fast as the round-robin baseline.                                                  */
+#define NUNA_HINT_RESIDENT    32u
+/* `flags`, bit 6: launch with programmatic stream serialization.  The kernel may be scheduled while its
+ * predecessor in the stream drains; it waits for that grid's completion and memory visibility before
+ * its first global access, so results are those of an ordinary stream-ordered launch.  Ignored by the
+ * flag-barrier two-shot (a cooperative launch) and above 16 MiB of sources, where it does not pay.     */
+#define NUNA_LAUNCH_PDL       64u
 
 /* Create the calling thread's current device's context (flag-barrier words, status word, work cursors,
  * two-shot shard scratch of `scratch_bytes`).  Called implicitly by the first collective on a device;
@@ -108,13 +118,26 @@ int nuna_allgather(const void* const* src, void* const* dst, int nranks,
 int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks,
                         size_t count, int dtype, unsigned flags, int two_shot);
 
+/* Decode-step chain: `nnodes` back-to-back allreduces (two per transformer layer) captured once into a
+ * CUDA graph and replayed with a single launch.  src_sets / dst_sets are HOST arrays of nsets*nranks
+ * device pointers, set s occupying entries [s*nranks, (s+1)*nranks); node k works on set k mod nsets
+ * and starts reading only after node k-1 has finished writing.  flags as for the allreduce calls
+ * (NUNA_LAUNCH_PDL overlaps each node's launch with its predecessor's drain); two_shot selects
+ * nuna_allreduce_twoshot.  Creation allocates and synchronises nothing on the caller's streams; the
+ * chain reads the buffers named at creation on every launch.  *chain_out is an opaque handle.          */
+int nuna_chain_create(const void* const* src_sets, void* const* dst_sets, int nsets, int nnodes, int nranks,
+                      size_t count, int dtype, unsigned flags, int two_shot, void** chain_out);
+int nuna_chain_launch(void* chain, void* stream);      /* one replay of all nodes, asynchronous on `stream` */
+int nuna_chain_destroy(void* chain);
+
 /* Reads and clears the device status word of the current device (NUNA_OK or NUNA_ERR_TIMEOUT) after
  * synchronising the device.  After a timeout the barrier words are re-initialised.                     */
 int nuna_device_status(int* out);
 
 /* Launches an empty kernel of `blocks` thread blocks with the collectives' block shape on `stream`: the
- * single-kernel-launch floor that small-message latencies are reported against.                        */
-int nuna_launch_floor(unsigned blocks, void* stream);
+ * single-kernel-launch floor that small-message latencies are reported against.  flags: 0 or
+ * NUNA_LAUNCH_PDL.                                                                                      */
+int nuna_launch_floor(unsigned blocks, unsigned flags, void* stream);
 
 /* Number of kernels this library has launched on any device since load (the callers' launch count).   */
 unsigned long long nuna_launch_count(void);

@@ -24,8 +24,10 @@ NUNA_BF16, NUNA_F16, NUNA_F32 = 0, 1, 2
 NUNA_MAX_RANKS = 16
 NUNA_PLACE_ROUNDROBIN, NUNA_PLACE_AWARE, NUNA_PLACE_AUTO = 0, 1, 2
 NUNA_TWOSHOT_PUT = 16
+NUNA_HINT_RESIDENT = 32
+NUNA_LAUNCH_PDL = 64
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libnuna.so")
+_LIB_PATH = os.environ.get("NUNA_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libnuna.so")
 _lib = None
 
 
@@ -54,8 +56,15 @@ def lib() -> ctypes.CDLL:
         L.nuna_init.restype = ctypes.c_int
         L.nuna_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
         L.nuna_device_status.restype = ctypes.c_int
-        L.nuna_launch_floor.argtypes = [ctypes.c_uint, ctypes.c_void_p]
+        L.nuna_launch_floor.argtypes = [ctypes.c_uint, ctypes.c_uint, ctypes.c_void_p]
         L.nuna_launch_floor.restype = ctypes.c_int
+        L.nuna_chain_create.argtypes = [vpp, vpp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_size_t, ctypes.c_int,
+                                        ctypes.c_uint, ctypes.c_int, ctypes.POINTER(ctypes.c_void_p)]
+        L.nuna_chain_create.restype = ctypes.c_int
+        L.nuna_chain_launch.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+        L.nuna_chain_launch.restype = ctypes.c_int
+        L.nuna_chain_destroy.argtypes = [ctypes.c_void_p]
+        L.nuna_chain_destroy.restype = ctypes.c_int
         L.nuna_launch_count.argtypes = []
         L.nuna_launch_count.restype = ctypes.c_ulonglong
         L.nuna_status_string.argtypes = [ctypes.c_int]
@@ -132,6 +141,26 @@ def nuna_allreduce_host(src, dst, count, dtype=NUNA_BF16, flags=0, two_shot=Fals
     return _finish(st, "nuna_allreduce_host", check)
 
 
+def nuna_chain_create(src_sets, dst_sets, nnodes, count, dtype=NUNA_BF16, flags=0, two_shot=False, check=True):
+    """``src_sets`` / ``dst_sets``: sequences (one per buffer set) of per-rank buffers.  Returns a handle."""
+    nsets, nranks = len(src_sets), len(src_sets[0])
+    flat_s = [b for s in src_sets for b in s]
+    flat_d = [b for s in dst_sets for b in s]
+    handle = ctypes.c_void_p()
+    st = lib().nuna_chain_create(ptr_table(flat_s), ptr_table(flat_d), nsets, nnodes, nranks, count, dtype, flags,
+                                 1 if two_shot else 0, ctypes.byref(handle))
+    _finish(st, "nuna_chain_create", check)
+    return handle if st == NUNA_OK else st
+
+
+def nuna_chain_launch(chain, stream=None, check=True) -> int:
+    return _finish(lib().nuna_chain_launch(chain, _stream(stream)), "nuna_chain_launch", check)
+
+
+def nuna_chain_destroy(chain) -> int:
+    return lib().nuna_chain_destroy(chain)
+
+
 def nuna_device_status() -> int:
     out = ctypes.c_int(0)
     st = lib().nuna_device_status(ctypes.byref(out))
@@ -140,8 +169,8 @@ def nuna_device_status() -> int:
     return out.value
 
 
-def nuna_launch_floor(blocks: int, stream=None, check: bool = True) -> int:
-    return _finish(lib().nuna_launch_floor(blocks, _stream(stream)), "nuna_launch_floor", check)
+def nuna_launch_floor(blocks: int, flags: int = 0, stream=None, check: bool = True) -> int:
+    return _finish(lib().nuna_launch_floor(blocks, flags, _stream(stream)), "nuna_launch_floor", check)
 
 
 def nuna_launch_count() -> int:

@@ -1,5 +1,6 @@
 // Host side of the C ABI: argument checks, per-device context, launch configuration.
 #include "nuna_internal.h"
+#include "nuna_kernels.cuh"
 
 #include <algorithm>
 #include <atomic>
@@ -44,6 +45,8 @@ int get_context(Context** out)
         c->timeout_ns = (unsigned long long)env_int("NUNA_TIMEOUT_MS", 1000) * 1000000ull;
         c->blocks_override = env_int("NUNA_BLOCKS", 0);
         c->unroll_override = env_int("NUNA_UNROLL", 0);
+        c->auto_min_bytes = (size_t)env_int("NUNA_AUTO_MIN_BYTES", 64 << 10);
+        c->coloc_override = env_int("NUNA_COLOC", 0);
         g_ctx[dev] = c;
     }
     *out = g_ctx[dev];
@@ -53,8 +56,6 @@ int get_context(Context** out)
 int ensure_scratch(Context* c, size_t bytes)
 {
     if (bytes <= c->scratch_bytes) return NUNA_OK;
-    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
-    (void)cs;
     void* p = nullptr;
     const size_t want = (bytes + 255) & ~(size_t)255;
     if (cudaMalloc(&p, want) != cudaSuccess) return NUNA_ERR_CUDA;
@@ -79,7 +80,8 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
     if (nranks < 1) return NUNA_ERR_INVALID_ARG;
     if (dtype != NUNA_BF16) return (dtype == NUNA_F16 || dtype == NUNA_F32) ? NUNA_ERR_UNSUPPORTED_DTYPE
                                                                              : NUNA_ERR_UNSUPPORTED_DTYPE;
-    if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT)) != 0u || (flags & NUNA_PLACE_MASK) == 3u)
+    if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT | NUNA_HINT_RESIDENT | NUNA_LAUNCH_PDL)) != 0u ||
+        (flags & NUNA_PLACE_MASK) == 3u)
         return NUNA_ERR_INVALID_ARG;
     if (src_elems > ((size_t)1 << 40) || dst_elems > ((size_t)1 << 40)) return NUNA_ERR_TOO_LARGE;
     if (src_elems == 0 && dst_elems == 0) return NUNA_OK;
@@ -140,20 +142,32 @@ static unsigned pick_grid(const Context* c, size_t nitems, int blocks_per_sm)
     return (unsigned)std::max<size_t>(1, std::min(nitems, cap));
 }
 
-template <typename... Args, typename... Act>
-static int launch(void (*kernel)(Args...), unsigned grid, cudaStream_t stream, bool cooperative, Act&&... args)
+constexpr unsigned kLaunchPlain = 0u, kLaunchCooperative = 1u, kLaunchPdl = 2u;
+
+// Programmatic dependent launch pays off while a kernel is short enough for its launch latency to
+// matter; from about 16 MiB of sources it was measured to cost a few percent, so it is dropped there.
+static unsigned launch_mode(unsigned flags, size_t total_src_bytes = 0)
 {
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof cfg);
+    return ((flags & NUNA_LAUNCH_PDL) && total_src_bytes <= ((size_t)16 << 20)) ? kLaunchPdl : kLaunchPlain;
+}
+
+template <typename... Args, typename... Act>
+static int launch(void (*kernel)(Args...), unsigned grid, cudaStream_t stream, unsigned mode, Act&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     int nattr = 0;
-    if (cooperative) {
+    if (mode & kLaunchCooperative) {
         attr[nattr].id = cudaLaunchAttributeCooperative;
         attr[nattr].val.cooperative = 1;
+        ++nattr;
+    } else if (mode & kLaunchPdl) {
+        attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[nattr].val.programmaticStreamSerializationAllowed = 1;
         ++nattr;
     }
     cfg.attrs = attr;
@@ -199,10 +213,47 @@ static size_t ceil_div(size_t a, size_t b) { return (a + b - 1) / b; }
 
 // ---- collectives ---------------------------------------------------------------------------------
 
+// NUNA_PLACE_AUTO: use the placement-aware kernel only where it is at least as fast as the
+// round-robin baseline.  NUNA_AUTO_MIN_BYTES overrides the measured crossover (bytes per rank).
+static bool aware_pays_off(const Context* c, int nranks, size_t count, unsigned flags)
+{
+    if (nranks < 2 || !(flags & NUNA_HINT_RESIDENT)) return false;
+    const size_t bytes = count * 2;
+    // sources and destinations of one call, twice over (the producer's other buffers), must fit in L2
+    // for "resident" to be physically possible
+    if (4 * bytes * (size_t)nranks > c->l2_bytes) return false;
+    return bytes >= c->auto_min_bytes;
+}
+
+
+template <int N, int C>
+static int launch_group(Context* c, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
+{
+    static int occ = 0;
+    auto k = k_oneshot_group<N, C>;
+    const size_t nvec = count / kVecElems;
+    const size_t ntiles = ceil_div(nvec, (size_t)(kThreads / C));
+    const size_t nitems = std::max<size_t>(ntiles * ((N + C - 1) / C), (count % kVecElems) ? (size_t)N : 0);
+    const unsigned grid = pick_grid(c, nitems, occupancy(c, k, &occ));
+    return launch(k, grid, stream, mode, p, count, ntiles);
+}
+
 int launch_oneshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream)
 {
-    (void)flags;
+    const unsigned mode = launch_mode(flags, count * 2 * (size_t)nranks);
     const size_t nvec = count / kVecElems;
+    const unsigned place = flags & NUNA_PLACE_MASK;
+    if (place == NUNA_PLACE_AWARE || (place == NUNA_PLACE_AUTO && aware_pays_off(c, nranks, count, flags))) {
+        // co-location factor: C destinations of a tile share a block (C <= N rounded up to a power of two)
+        int coloc = c->coloc_override > 0 ? c->coloc_override : 8;
+        while (coloc > 1 && coloc / 2 >= nranks) coloc >>= 1;
+        return dispatch(nranks, 1, [&](auto n_, auto) -> int {
+            constexpr int N = decltype(n_)::value;
+            if (coloc >= 8) return launch_group<N, 8>(c, p, count, mode, stream);
+            if (coloc >= 4) return launch_group<N, 4>(c, p, count, mode, stream);
+            return launch_group<N, 2>(c, p, count, mode, stream);
+        });
+    }
     return dispatch(nranks, pick_unroll(c, nranks), [&](auto n_, auto u_) -> int {
         NUNA_NU(n_, u_);
         static int occ = 0;
@@ -210,12 +261,13 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsi
         const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
         const size_t nitems = std::max<size_t>(ntiles * N, (count % kVecElems) ? (size_t)N : 0);
         const unsigned grid = pick_grid(c, nitems, occupancy(c, k, &occ));
-        return launch(k, grid, stream, false, p, count, ntiles);
+        return launch(k, grid, stream, mode, p, count, ntiles);
     });
 }
 
 int launch_twoshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream)
 {
+    const unsigned mode = launch_mode(flags, count * 2 * (size_t)nranks);
     const size_t nvec = count / kVecElems;
     if (flags & NUNA_TWOSHOT_PUT) {
         return dispatch(nranks, pick_unroll(c, nranks), [&](auto n_, auto u_) -> int {
@@ -224,7 +276,7 @@ int launch_twoshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsi
             auto k = k_twoshot_put<N, U>;
             const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
             const unsigned grid = pick_grid(c, std::max<size_t>(ntiles, 1), occupancy(c, k, &occ));
-            return launch(k, grid, stream, false, p, count, ntiles);
+            return launch(k, grid, stream, mode, p, count, ntiles);
         });
     }
     // chunk = ceil(count / N) rounded up to whole vectors
@@ -238,18 +290,19 @@ int launch_twoshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsi
         size_t cap = (size_t)c->num_sms * (size_t)occupancy(c, k, &occ);
         if (c->blocks_override > 0) cap = std::min<size_t>(cap, (size_t)c->blocks_override);
         const unsigned grid = (unsigned)std::max<size_t>(1, std::min(tiles_per_chunk * N, cap));
-        return launch(k, grid, stream, true, p, reinterpret_cast<uint4*>(c->scratch), count, chunk_vec,
+        return launch(k, grid, stream, kLaunchCooperative, p, reinterpret_cast<uint4*>(c->scratch), count, chunk_vec,
                       c->bw, c->timeout_ns);
     });
 }
 
-int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shard, cudaStream_t stream)
+int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shard, unsigned flags, cudaStream_t stream)
 {
+    const unsigned mode = launch_mode(flags);
     if (shard % kVecElems) {
         const unsigned grid = pick_grid(c, ceil_div(shard * nranks, kThreads), 8);
         return dispatch(nranks, 1, [&](auto n_, auto u_) -> int {
             NUNA_NU(n_, u_);
-            return launch(k_reduce_scatter_scalar<N>, grid, stream, false, p, shard);
+            return launch(k_reduce_scatter_scalar<N>, grid, stream, mode, p, shard);
         });
     }
     const size_t shard_vec = shard / kVecElems;
@@ -259,15 +312,16 @@ int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shar
         auto k = k_reduce_scatter<N, U>;
         const size_t tiles = ceil_div(shard_vec, (size_t)kThreads * U);
         const unsigned grid = pick_grid(c, tiles * N, occupancy(c, k, &occ));
-        return launch(k, grid, stream, false, p, shard_vec, tiles);
+        return launch(k, grid, stream, mode, p, shard_vec, tiles);
     });
 }
 
-int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, cudaStream_t stream)
+int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, unsigned flags, cudaStream_t stream)
 {
+    const unsigned mode = launch_mode(flags);
     if (shard % kVecElems) {
         const unsigned grid = pick_grid(c, ceil_div(shard * nranks, kThreads), 8);
-        return launch(k_allgather_scalar, grid, stream, false, p, nranks, shard);
+        return launch(k_allgather_scalar, grid, stream, mode, p, nranks, shard);
     }
     const size_t shard_vec = shard / kVecElems;
     static int occ = 0;
@@ -275,7 +329,7 @@ int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, cu
     auto k = k_allgather<U>;
     const size_t tiles = ceil_div(shard_vec, (size_t)kThreads * U);
     const unsigned grid = pick_grid(c, tiles * nranks, occupancy(c, k, &occ));
-    return launch(k, grid, stream, false, p, nranks, shard_vec, tiles);
+    return launch(k, grid, stream, mode, p, nranks, shard_vec, tiles);
 }
 
 }  // namespace nuna
@@ -335,7 +389,7 @@ int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks, si
     if (flags & NUNA_TWOSHOT_PUT) return NUNA_ERR_INVALID_ARG;
     Context* c = nullptr;
     if ((st = get_context(&c)) != NUNA_OK) return st;
-    return launch_reduce_scatter(c, make_ptrs(src, dst, nranks), nranks, shard_count, (cudaStream_t)stream);
+    return launch_reduce_scatter(c, make_ptrs(src, dst, nranks), nranks, shard_count, flags, (cudaStream_t)stream);
 }
 
 int nuna_allgather(const void* const* src, void* const* dst, int nranks, size_t shard_count, int dtype,
@@ -349,7 +403,7 @@ int nuna_allgather(const void* const* src, void* const* dst, int nranks, size_t 
     if (flags & NUNA_TWOSHOT_PUT) return NUNA_ERR_INVALID_ARG;
     Context* c = nullptr;
     if ((st = get_context(&c)) != NUNA_OK) return st;
-    return launch_allgather(c, make_ptrs(src, dst, nranks), nranks, shard_count, (cudaStream_t)stream);
+    return launch_allgather(c, make_ptrs(src, dst, nranks), nranks, shard_count, flags, (cudaStream_t)stream);
 }
 
 int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
@@ -406,10 +460,10 @@ int nuna_device_status(int* out)
     return NUNA_OK;
 }
 
-int nuna_launch_floor(unsigned blocks, void* stream)
+int nuna_launch_floor(unsigned blocks, unsigned flags, void* stream)
 {
-    if (blocks == 0 || blocks > (1u << 20)) return NUNA_ERR_INVALID_ARG;
-    return launch(k_empty, blocks, (cudaStream_t)stream, false, 0);
+    if (blocks == 0 || blocks > (1u << 20) || (flags & ~NUNA_LAUNCH_PDL)) return NUNA_ERR_INVALID_ARG;
+    return launch(k_empty, blocks, (cudaStream_t)stream, launch_mode(flags), 0);
 }
 
 unsigned long long nuna_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
@@ -461,7 +515,7 @@ int nuna_debug_barrier_selftest(unsigned grid, unsigned expected, unsigned timeo
     unsigned* d = nullptr;
     if (cudaMalloc(&d, sizeof(unsigned)) != cudaSuccess) return NUNA_ERR_CUDA;
     cudaMemset(d, 0, sizeof(unsigned));
-    st = launch(k_barrier_selftest, grid, (cudaStream_t)0, true, c->bw, expected,
+    st = launch(k_barrier_selftest, grid, (cudaStream_t)0, kLaunchCooperative, c->bw, expected,
                 (unsigned long long)timeout_ms * 1000000ull, d);
     if (st == NUNA_OK && cudaDeviceSynchronize() != cudaSuccess) st = NUNA_ERR_CUDA;
     if (st == NUNA_OK && cudaMemcpy(passed, d, sizeof(unsigned), cudaMemcpyDeviceToHost) != cudaSuccess) st = NUNA_ERR_CUDA;

@@ -6,7 +6,7 @@
 #include <mutex>
 
 #include "../../include/nuna.h"
-#include "nuna_kernels.cuh"
+#include "nuna_types.h"
 
 namespace nuna {
 
@@ -25,6 +25,8 @@ struct Context {
     unsigned long long timeout_ns = 1000000000ull;
     int blocks_override = 0;             // NUNA_BLOCKS
     int unroll_override = 0;             // NUNA_UNROLL
+    int coloc_override = 0;              // NUNA_COLOC: destinations of a tile per block (2, 4, 8)
+    size_t auto_min_bytes = 0;           // NUNA_PLACE_AUTO picks the aware kernel from this size per rank
     std::mutex mutex;
 };
 
@@ -36,7 +38,7 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
                int dtype, unsigned flags, bool device_ptrs);
 int launch_oneshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream);
 int launch_twoshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream);
-int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shard, cudaStream_t stream);
-int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, cudaStream_t stream);
+int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shard, unsigned flags, cudaStream_t stream);
+int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, unsigned flags, cudaStream_t stream);
 
 }  // namespace nuna

@@ -9,11 +9,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "nuna_types.h"
+
 namespace nuna {
 
-constexpr int kMaxRanks = 16;
-constexpr int kThreads = 256;            // threads per block, every kernel
-constexpr int kVecElems = 8;             // bf16 per 16-byte vector
 
 // Blocks per SM the compiler is asked to keep resident for a kernel that holds `vectors` 16-byte
 // loads in flight per thread.  Stating it makes ptxas spend registers on keeping ALL of a thread's
@@ -26,10 +25,27 @@ constexpr int min_blocks(int vectors)
     return b < 1 ? 1 : (b > 8 ? 8 : b);
 }
 
-struct RankPtrs {
-    const uint4* src[kMaxRanks];
-    uint4* dst[kMaxRanks];
-};
+
+// ---- programmatic dependent launch ---------------------------------------------------------------
+//
+// Every collective kernel opens with pdl_wait() and calls pdl_trigger() when its block has issued
+// its main work.  When a kernel is launched with programmatic stream serialization
+// (NUNA_LAUNCH_PDL) its blocks may be scheduled while the predecessor in the stream drains:
+// griddepcontrol.wait holds them, before their first global access, until the predecessor grid has
+// completed and its memory operations are visible; griddepcontrol.launch_dependents, issued once a
+// block is past its main loop, lets the successor's blocks take the freed SM slots so that their
+// launch latency overlaps this kernel's tail.  (Triggering at kernel entry instead was measured
+// slower: the successor's waiting blocks then compete with this kernel's own blocks for slots.)
+// Launched normally, both instructions do nothing.
+__device__ __forceinline__ void pdl_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+__device__ __forceinline__ void pdl_trigger()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
 // ---- memory access helpers ----------------------------------------------------------------
 
@@ -67,23 +83,25 @@ __device__ __forceinline__ uint16_t ld_src16(const uint16_t* p)
 
 // ---- the fold ------------------------------------------------------------------------------
 
-// bf16 -> binary32 is a 16-bit shift; a 32-bit word holds elements (2k) in its low half and
-// (2k+1) in its high half.
-__device__ __forceinline__ void widen(float (&a)[8], uint4 v)
+// bf16 -> binary32 is a 16-bit shift; a 32-bit word holds element 2k in its low half and 2k+1
+// in its high half.  Rank 0's value is widened with a shift / mask; ranks 1..N-1 are folded in with
+// the sm_100 mixed-precision add, d = f32(bf16 a) + c rounded once to binary32 (nearest even,
+// subnormals kept), so no instruction is spent on widening them.  At large sizes the one-shot is
+// limited by instruction issue and L1 throughput (N times the work of a plain sum), which is why
+// the instruction count matters.
+__device__ __forceinline__ float add_bf16(float acc, uint16_t h)
 {
-    a[0] = __uint_as_float(v.x << 16); a[1] = __uint_as_float(v.x & 0xFFFF0000u);
-    a[2] = __uint_as_float(v.y << 16); a[3] = __uint_as_float(v.y & 0xFFFF0000u);
-    a[4] = __uint_as_float(v.z << 16); a[5] = __uint_as_float(v.z & 0xFFFF0000u);
-    a[6] = __uint_as_float(v.w << 16); a[7] = __uint_as_float(v.w & 0xFFFF0000u);
+    float d;
+    asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(acc));
+    return d;
 }
 
-// acc <- acc + f(v), IEEE add.rn.f32 (no flush-to-zero: the file is compiled without fast-math).
-__device__ __forceinline__ void fold_in(float (&a)[8], uint4 v)
+__device__ __forceinline__ void fold_word(float& lo, float& hi, uint32_t w)
 {
-    a[0] = __fadd_rn(a[0], __uint_as_float(v.x << 16)); a[1] = __fadd_rn(a[1], __uint_as_float(v.x & 0xFFFF0000u));
-    a[2] = __fadd_rn(a[2], __uint_as_float(v.y << 16)); a[3] = __fadd_rn(a[3], __uint_as_float(v.y & 0xFFFF0000u));
-    a[4] = __fadd_rn(a[4], __uint_as_float(v.z << 16)); a[5] = __fadd_rn(a[5], __uint_as_float(v.z & 0xFFFF0000u));
-    a[6] = __fadd_rn(a[6], __uint_as_float(v.w << 16)); a[7] = __fadd_rn(a[7], __uint_as_float(v.w & 0xFFFF0000u));
+    uint16_t l, h;
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(l), "=h"(h) : "r"(w));
+    lo = add_bf16(lo, l);
+    hi = add_bf16(hi, h);
 }
 
 // Two binary32 -> one word of two bf16, round to nearest even, NaN -> 0x7FFF.
@@ -94,20 +112,23 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
     return d;
 }
 
-__device__ __forceinline__ uint4 narrow(const float (&a)[8])
-{
-    return make_uint4(pack2(a[0], a[1]), pack2(a[2], a[3]), pack2(a[4], a[5]), pack2(a[6], a[7]));
-}
-
-// Fold N already-loaded vectors in rank order.
+// Fold N already-loaded vectors in rank order: acc starts from rank 0's value, N-1 additions.
 template <int N>
 __device__ __forceinline__ uint4 fold_vectors(const uint4 (&v)[N])
 {
     float a[8];
-    widen(a, v[0]);
+    a[0] = __uint_as_float(v[0].x << 16); a[1] = __uint_as_float(v[0].x & 0xFFFF0000u);
+    a[2] = __uint_as_float(v[0].y << 16); a[3] = __uint_as_float(v[0].y & 0xFFFF0000u);
+    a[4] = __uint_as_float(v[0].z << 16); a[5] = __uint_as_float(v[0].z & 0xFFFF0000u);
+    a[6] = __uint_as_float(v[0].w << 16); a[7] = __uint_as_float(v[0].w & 0xFFFF0000u);
 #pragma unroll
-    for (int r = 1; r < N; ++r) fold_in(a, v[r]);
-    return narrow(a);
+    for (int r = 1; r < N; ++r) {
+        fold_word(a[0], a[1], v[r].x);
+        fold_word(a[2], a[3], v[r].y);
+        fold_word(a[4], a[5], v[r].z);
+        fold_word(a[6], a[7], v[r].w);
+    }
+    return make_uint4(pack2(a[0], a[1]), pack2(a[2], a[3]), pack2(a[4], a[5]), pack2(a[6], a[7]));
 }
 
 // One element (ragged tails and unaligned shards).
@@ -151,11 +172,70 @@ template <int N, int U>
 __global__ void __launch_bounds__(kThreads, min_blocks(N * U))
 k_oneshot_rr(const RankPtrs p, const size_t count, const size_t ntiles)
 {
+    pdl_wait();
     const size_t nvec = count / kVecElems;
     const size_t nitems = ntiles * N;
     for (size_t item = blockIdx.x; item < nitems; item += gridDim.x)
         oneshot_item<N, U>(p, nvec, item / N, (int)(item % N));
+    pdl_trigger();
     // ragged tail (count % 8 elements): block d handles destination d
+    const size_t tail0 = nvec * kVecElems;
+    if (tail0 < count) {
+        for (int d = blockIdx.x; d < N; d += gridDim.x) {
+            const size_t e = tail0 + threadIdx.x;
+            if (e < count) reinterpret_cast<uint16_t*>(p.dst[d])[e] = fold_scalar<N>(p, e);
+        }
+    }
+}
+
+// ---- one-shot allreduce, co-located groups (placement-aware) ------------------------------------------
+//
+// Logical allocation (Section 4.2.1) puts the thread blocks that touch the same chunks into
+// one group, and physical placement keeps a group on one compute unit.  For the one-shot the N
+// work items (tile, d), d = 0..N-1, share all N source tiles, so a group is "one tile, every
+// destination".  Here a group runs inside ONE thread block: row d of the block (kThreads / rows
+// threads, rows = N rounded up to a power of two) is emulated rank d's work item for that tile.
+// Every row still issues its own loads of all N sources and does its own fold, but the rows'
+// requests for the same lines meet in that SM's L1, so each source line crosses the L2 -> SM
+// fabric once per group instead of once per destination.
+__device__ __forceinline__ uint4 ld_src_l1(const uint4* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// Co-location factor C (a power of two, at most N rounded up to one): a block holds the work items
+// of C destinations of one tile, so a tile's group is spread over ceil(N / C) blocks.  This is the
+// resource budget of Section 4.2.2 in SM terms: the more items of a group share an SM, the fewer
+// distinct bytes that SM has in flight (kThreads / C vectors per source), so cold data wants a small
+// C (more outstanding requests per SM) and L2-resident data a large one (fewer L2 -> SM transfers).
+template <int N, int C>
+__device__ __forceinline__ void oneshot_group(const RankPtrs& p, size_t nvec, size_t tile, int dst0)
+{
+    constexpr int kLanes = kThreads / C;                 // vectors per tile
+    const int d = dst0 + threadIdx.x / kLanes;
+    const size_t i = tile * kLanes + (threadIdx.x % kLanes);
+    if (d < N && i < nvec) {
+        uint4 v[N];
+#pragma unroll
+        for (int r = 0; r < N; ++r) v[r] = ld_src_l1(p.src[r] + i);
+        st_dst(p.dst[d] + i, fold_vectors<N>(v));
+    }
+}
+
+template <int N, int C>
+__global__ void __launch_bounds__(kThreads, min_blocks(N))
+k_oneshot_group(const RankPtrs p, const size_t count, const size_t ntiles)
+{
+    pdl_wait();
+    constexpr int kSplit = (N + C - 1) / C;              // blocks per tile group
+    const size_t nvec = count / kVecElems;
+    const size_t nitems = ntiles * kSplit;
+    for (size_t it = blockIdx.x; it < nitems; it += gridDim.x)
+        oneshot_group<N, C>(p, nvec, it / kSplit, (int)(it % kSplit) * C);
+    pdl_trigger();
     const size_t tail0 = nvec * kVecElems;
     if (tail0 < count) {
         for (int d = blockIdx.x; d < N; d += gridDim.x) {
@@ -194,12 +274,14 @@ template <int N, int U>
 __global__ void __launch_bounds__(kThreads, min_blocks(N * U))
 k_reduce_scatter(const RankPtrs p, const size_t shard_vec, const size_t tiles_per_shard)
 {
+    pdl_wait();
     const size_t nitems = tiles_per_shard * N;
     for (size_t item = blockIdx.x; item < nitems; item += gridDim.x) {
         const int r = (int)(item / tiles_per_shard);
         const size_t tile = item % tiles_per_shard;
         reduce_tile<N, U>(p, p.dst[r], (size_t)r * shard_vec, shard_vec, tile);
     }
+    pdl_trigger();
 }
 
 // Any shard length: one element per thread (slow path, used when S % 8 != 0).
@@ -207,6 +289,7 @@ template <int N>
 __global__ void __launch_bounds__(kThreads)
 k_reduce_scatter_scalar(const RankPtrs p, const size_t shard)
 {
+    pdl_wait();
     const size_t total = shard * N;
     for (size_t e = (size_t)blockIdx.x * kThreads + threadIdx.x; e < total; e += (size_t)gridDim.x * kThreads) {
         const int r = (int)(e / shard);
@@ -239,17 +322,20 @@ template <int U>
 __global__ void __launch_bounds__(kThreads, min_blocks(U))
 k_allgather(const RankPtrs p, const int nranks, const size_t shard_vec, const size_t tiles_per_shard)
 {
+    pdl_wait();
     const size_t nitems = tiles_per_shard * nranks;
     for (size_t item = blockIdx.x; item < nitems; item += gridDim.x) {
         const int r = (int)(item / tiles_per_shard);
         const size_t tile = item % tiles_per_shard;
         gather_tile<U>(p.src[r], p, nranks, (size_t)r * shard_vec, shard_vec, tile, false);
     }
+    pdl_trigger();
 }
 
 __global__ void __launch_bounds__(kThreads)
 k_allgather_scalar(const RankPtrs p, const int nranks, const size_t shard)
 {
+    pdl_wait();
     const size_t total = shard * nranks;
     for (size_t e = (size_t)blockIdx.x * kThreads + threadIdx.x; e < total; e += (size_t)gridDim.x * kThreads) {
         const int r = (int)(e / shard);
@@ -267,12 +353,6 @@ k_allgather_scalar(const RankPtrs p, const int nranks, const size_t shard)
 // grows, so graph replays need no host reset.  Every wait is bounded: after
 // `timeout_ns` the block latches NUNA_ERR_TIMEOUT in `status` and returns false;
 // the caller then skips the rest of its work and exits.  Nothing traps or hangs.
-struct BarrierWords {
-    unsigned int arrive;
-    unsigned int epoch;
-    unsigned int status;
-    unsigned int pad;
-};
 
 __device__ __forceinline__ unsigned long long globaltimer_ns()
 {
@@ -376,6 +456,7 @@ template <int N, int U>
 __global__ void __launch_bounds__(kThreads, min_blocks(N * U))
 k_twoshot_put(const RankPtrs p, const size_t count, const size_t ntiles)
 {
+    pdl_wait();
     const size_t nvec = count / kVecElems;
     for (size_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const size_t base = tile * (size_t)(kThreads * U) + threadIdx.x;
@@ -398,6 +479,7 @@ k_twoshot_put(const RankPtrs p, const size_t count, const size_t ntiles)
             }
         }
     }
+    pdl_trigger();
     const size_t tail0 = nvec * kVecElems;
     if (tail0 < count && blockIdx.x == 0) {
         const size_t e = tail0 + threadIdx.x;
@@ -418,6 +500,6 @@ __global__ void k_barrier_selftest(BarrierWords* bw, unsigned int expected, unsi
 }
 
 // Launch-floor reference: same grid shape, no memory traffic.
-__global__ void __launch_bounds__(kThreads) k_empty(int) {}
+__global__ void __launch_bounds__(kThreads) k_empty(int) { pdl_wait(); pdl_trigger(); }
 
 }  // namespace nuna

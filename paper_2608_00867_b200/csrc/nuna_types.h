@@ -1,0 +1,26 @@
+// Plain types shared by the library's host code and its kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace nuna {
+
+constexpr int kMaxRanks = 16;
+constexpr int kThreads = 256;            // threads per block, every kernel
+constexpr int kVecElems = 8;             // bf16 per 16-byte vector
+
+// Kernel argument: the rank buffers, by value.
+struct RankPtrs {
+    const uint4* src[kMaxRanks];
+    uint4* dst[kMaxRanks];
+};
+
+// Flag-barrier words and the latched device status, in device memory.
+struct BarrierWords {
+    unsigned int arrive;
+    unsigned int epoch;
+    unsigned int status;
+    unsigned int pad;
+};
+
+}  // namespace nuna

@@ -58,7 +58,7 @@ COUNTS = [1, 7, 8, 9, 15, 16, 17, 2047, 2048, 2049, 4096, 6151, 100003, 262144]
 
 
 @pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16])
-@pytest.mark.parametrize("algo", ["oneshot", "twoshot", "twoshot_put"])
+@pytest.mark.parametrize("algo", ["oneshot", "oneshot_aware", "twoshot", "twoshot_put"])
 def test_allreduce_special_values_all_counts(n, algo):
     for count in COUNTS:
         src = workloads.special_values(n, count, seed=1000 * n + count % 997)
@@ -66,6 +66,8 @@ def test_allreduce_special_values_all_counts(n, algo):
         dsrc, dst = upload(src), Dst(n, count)
         if algo == "oneshot":
             nb.nuna_allreduce_oneshot(dsrc, dst.view, count)
+        elif algo == "oneshot_aware":
+            nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE)
         else:
             nb.nuna_allreduce_twoshot(dsrc, dst.view, count, flags=nb.NUNA_TWOSHOT_PUT if algo == "twoshot_put" else 0)
         got = dst.numpy()
@@ -142,8 +144,8 @@ def test_sweep_sizes_one_and_two_shot_agree_with_oracle():
         src = workloads.make(w)
         want = oracle.allreduce(src, nthreads=8)[0]
         dsrc = upload(src)
-        for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_twoshot, 0),
-                            (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
+        for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE),
+                            (nb.nuna_allreduce_twoshot, 0), (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
             dst = Dst(w.nranks, w.count)
             call(dsrc, dst.view, w.count, flags=flags)
             got = dst.numpy()
@@ -170,8 +172,8 @@ def test_full_size_64MiB_sampled_columns_and_invariants():
     cols = np.stack([t[tidx].cpu().numpy().view(np.uint16) for t in dsrc])          # [n, len(idx)]
     want = oracle.allreduce([np.ascontiguousarray(c) for c in cols], nthreads=4)[0]
     results = []
-    for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_twoshot, 0),
-                        (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
+    for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE),
+                        (nb.nuna_allreduce_twoshot, 0), (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
         dst = [torch.full((count,), -1, dtype=torch.int16, device="cuda") for _ in range(n)]
         call(dsrc, dst, count, flags=flags)
         torch.cuda.synchronize()
@@ -180,7 +182,7 @@ def test_full_size_64MiB_sampled_columns_and_invariants():
             assert torch.equal(dst[0], dst[d])                        # all destinations identical
         results.append(dst[0].clone())
         del dst
-    assert torch.equal(results[0], results[1]) and torch.equal(results[0], results[2])
+    assert all(torch.equal(results[0], r) for r in results[1:])
     assert nb.nuna_device_status() == nb.NUNA_OK
 
 
@@ -204,6 +206,56 @@ def test_graph_replay_gives_same_bits():
         torch.cuda.synchronize()
         for t in dst:
             assert np.array_equal(t.cpu().numpy().view(np.uint16), want)
+
+
+@pytest.mark.parametrize("flags", [0, nb.NUNA_LAUNCH_PDL, nb.NUNA_LAUNCH_PDL | nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT])
+@pytest.mark.parametrize("two_shot", [False, True])
+def test_chain_every_node_matches_oracle(flags, two_shot):
+    tokens = 8
+    w = workloads.config_decode_chain(tokens)
+    nsets, nnodes = 2, 6
+    srcs = [workloads.rank_buffers(w.nranks, w.count, "normal", seed=w.seed + s) for s in range(nsets)]
+    want = [oracle.allreduce(s, nthreads=4)[0] for s in srcs]
+    dsrc = [upload(s) for s in srcs]
+    ddst = [[torch.zeros(w.count, dtype=torch.int16, device="cuda") for _ in range(w.nranks)] for _ in range(nsets)]
+    chain = nb.nuna_chain_create(dsrc, ddst, nnodes, w.count, flags=flags, two_shot=two_shot)
+    try:
+        for _ in range(3):
+            for dset in ddst:
+                for t in dset:
+                    t.zero_()
+            nb.nuna_chain_launch(chain)
+            torch.cuda.synchronize()
+            for s in range(nsets):
+                for t in ddst[s]:
+                    assert np.array_equal(t.cpu().numpy().view(np.uint16), want[s])
+    finally:
+        nb.nuna_chain_destroy(chain)
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
+@pytest.mark.parametrize("flags", [0, nb.NUNA_LAUNCH_PDL, nb.NUNA_LAUNCH_PDL | nb.NUNA_PLACE_AWARE])
+def test_chain_nodes_are_ordered_even_with_dependent_launch(flags):
+    """Node k+1 reads what node k wrote: ones -> 8 -> 64 -> 512 -> 4096 only if every node waited."""
+    n, count, levels = 8, 1 << 20, 4
+    one = np.int16(0x3F80)
+    bufs = [[torch.full((count,), one, dtype=torch.int16, device="cuda") for _ in range(n)]]
+    for _ in range(levels):
+        bufs.append([torch.zeros(count, dtype=torch.int16, device="cuda") for _ in range(n)])
+    chain = nb.nuna_chain_create(bufs[:-1], bufs[1:], levels, count, flags=flags)
+    try:
+        for _ in range(5):
+            for lvl in bufs[1:]:
+                for t in lvl:
+                    t.zero_()
+            nb.nuna_chain_launch(chain)
+            torch.cuda.synchronize()
+            for lvl, expect in zip(bufs[1:], (8.0, 64.0, 512.0, 4096.0)):
+                for t in lvl:
+                    v = t.view(torch.bfloat16)
+                    assert float(v.min()) == expect and float(v.max()) == expect
+    finally:
+        nb.nuna_chain_destroy(chain)
 
 
 def test_host_buffer_entry_point():
