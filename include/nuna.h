@@ -80,6 +80,54 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* on
  * flag-barrier two-shot (a cooperative launch) and above 16 MiB of sources, where it does not pay.     */
 #define NUNA_LAUNCH_PDL       64u
 
+/* ---- topology probe --------------------------------------------------------------------------------
+ * Result of nuna_probe_topology: caller-owned, plain data, fixed maximum sizes.  Latencies are in SM
+ * clock cycles per dependent load.  Entries for SMs that did not report are zero.                      */
+#define NUNA_MAX_SMS          256
+#define NUNA_MAX_PROBE_BUFS   32
+#define NUNA_PROBE_REGIONS    8
+#define NUNA_MAX_PROBE_LINES  2048
+#define NUNA_TOPO_UNIFORM     0
+#define NUNA_TOPO_NONUNIFORM  1
+
+typedef struct nuna_topology {
+    int num_sms;                     /* cudaDeviceProp.multiProcessorCount                                 */
+    int sms_reported;                /* SMs that ran a probe block (one block per SM is requested)         */
+    int num_bufs, num_regions;       /* buffers probed; each is cut into num_regions equal regions         */
+    int num_lines;                   /* 128-byte lines sampled in total                                    */
+    int num_domains;                 /* 1 = uniform; 2 = the SMs split into a near and a far side           */
+    int verdict;                     /* NUNA_TOPO_UNIFORM / NUNA_TOPO_NONUNIFORM                           */
+    int chain_nodes, chain_steps;    /* miss walk: nodes of the single-cycle permutation, steps per SM     */
+    int chain_walk_ok;               /* 1 if every SM's device walk ended on the node the host walk predicts */
+    int self_pointer_mismatches;     /* hit walk sanity: loads that did not return the line's own address   */
+    float nonuniformity;             /* (max - min) / min of the per-SM mean hit latencies                  */
+    float noise;                     /* median |repetition 0 - repetition 1| over all (SM, line) pairs      */
+    float near_lat, far_lat;         /* mean hit latency to lines at home in the SM's own / other domain    */
+    float domain_gap;                /* far_lat - near_lat                                                   */
+    int sm_reported[NUNA_MAX_SMS];
+    int sm_domain[NUNA_MAX_SMS];     /* 0 or 1; SM 0's side is domain 0; all 0 when uniform                  */
+    float sm_lat_hit[NUNA_MAX_SMS];  /* mean L2-hit latency of this SM over all sampled lines               */
+    float sm_lat_miss[NUNA_MAX_SMS]; /* mean latency of this SM's cold (DRAM) walk                           */
+    float lat_hit[NUNA_MAX_SMS][NUNA_MAX_PROBE_BUFS];               /* mean hit latency, SM x buffer          */
+    float region_home0[NUNA_MAX_PROBE_BUFS][NUNA_PROBE_REGIONS];    /* share of the region's sampled lines
+                                                                       that domain 0 reaches faster; -1 none */
+    unsigned char line_buf[NUNA_MAX_PROBE_LINES];                   /* per sampled line: buffer, region,      */
+    unsigned char line_region[NUNA_MAX_PROBE_LINES];                /* and the domain that reaches it faster  */
+    unsigned char line_home[NUNA_MAX_PROBE_LINES];
+} nuna_topology_t;
+
+/* Measures, for every SM (indexed by %smid) and every buffer, the latency of dependent L2-only loads
+ * to sampled lines of the caller's buffers (the analogue of the paper's per-compute-unit, per-address
+ * remote-access sweep, Section 3.2), plus each SM's cold DRAM latency, clusters the SMs into domains
+ * and stores the result in *out and in the device context (where NUNA_PLACE_AWARE plans read it).
+ * bufs: HOST array of nbufs (<= NUNA_MAX_PROBE_BUFS) device pointers, bytes[b] >= 128 each, 16-byte
+ * aligned.  One 8-byte word per sampled line is overwritten during the measurement and restored
+ * before return; the buffers must not be in use by other work meanwhile.  Synchronises `stream`,
+ * allocates temporary device memory (about 2.3 x the L2 size): NUNA_ERR_CAPTURING on a capturing
+ * stream.  Latency values are hardware facts and carry no parity claim.                               */
+int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
+                        nuna_topology_t* out, void* stream);
+
 /* Create the calling thread's current device's context (flag-barrier words, status word, work cursors,
  * two-shot shard scratch of `scratch_bytes`).  Called implicitly by the first collective on a device;
  * call it explicitly before stream capture, because it allocates.  Growing the scratch later also

@@ -27,6 +27,32 @@ NUNA_TWOSHOT_PUT = 16
 NUNA_HINT_RESIDENT = 32
 NUNA_LAUNCH_PDL = 64
 
+NUNA_MAX_SMS, NUNA_MAX_PROBE_BUFS, NUNA_PROBE_REGIONS, NUNA_MAX_PROBE_LINES = 256, 32, 8, 2048
+NUNA_TOPO_UNIFORM, NUNA_TOPO_NONUNIFORM = 0, 1
+
+
+class NunaTopology(ctypes.Structure):
+    """Mirror of ``nuna_topology_t`` (include/nuna.h)."""
+    _fields_ = [
+        ("num_sms", ctypes.c_int), ("sms_reported", ctypes.c_int),
+        ("num_bufs", ctypes.c_int), ("num_regions", ctypes.c_int), ("num_lines", ctypes.c_int),
+        ("num_domains", ctypes.c_int), ("verdict", ctypes.c_int),
+        ("chain_nodes", ctypes.c_int), ("chain_steps", ctypes.c_int), ("chain_walk_ok", ctypes.c_int),
+        ("self_pointer_mismatches", ctypes.c_int),
+        ("nonuniformity", ctypes.c_float), ("noise", ctypes.c_float),
+        ("near_lat", ctypes.c_float), ("far_lat", ctypes.c_float), ("domain_gap", ctypes.c_float),
+        ("sm_reported", ctypes.c_int * NUNA_MAX_SMS),
+        ("sm_domain", ctypes.c_int * NUNA_MAX_SMS),
+        ("sm_lat_hit", ctypes.c_float * NUNA_MAX_SMS),
+        ("sm_lat_miss", ctypes.c_float * NUNA_MAX_SMS),
+        ("lat_hit", (ctypes.c_float * NUNA_MAX_PROBE_BUFS) * NUNA_MAX_SMS),
+        ("region_home0", (ctypes.c_float * NUNA_PROBE_REGIONS) * NUNA_MAX_PROBE_BUFS),
+        ("line_buf", ctypes.c_ubyte * NUNA_MAX_PROBE_LINES),
+        ("line_region", ctypes.c_ubyte * NUNA_MAX_PROBE_LINES),
+        ("line_home", ctypes.c_ubyte * NUNA_MAX_PROBE_LINES),
+    ]
+
+
 _LIB_PATH = os.environ.get("NUNA_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libnuna.so")
 _lib = None
 
@@ -65,6 +91,15 @@ def lib() -> ctypes.CDLL:
         L.nuna_chain_launch.restype = ctypes.c_int
         L.nuna_chain_destroy.argtypes = [ctypes.c_void_p]
         L.nuna_chain_destroy.restype = ctypes.c_int
+        L.nuna_probe_topology.argtypes = [vpp, ctypes.POINTER(ctypes.c_size_t), ctypes.c_int,
+                                          ctypes.POINTER(NunaTopology), ctypes.c_void_p]
+        L.nuna_probe_topology.restype = ctypes.c_int
+        L.nuna_debug_analyse_topology.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
+                                                  ctypes.c_int, ctypes.c_int, ctypes.POINTER(NunaTopology)]
+        L.nuna_debug_analyse_topology.restype = ctypes.c_int
+        L.nuna_debug_chain.argtypes = [ctypes.POINTER(ctypes.c_uint), ctypes.c_int, ctypes.c_ulonglong, ctypes.c_uint,
+                                       ctypes.c_int, ctypes.POINTER(ctypes.c_uint)]
+        L.nuna_debug_chain.restype = ctypes.c_int
         L.nuna_launch_count.argtypes = []
         L.nuna_launch_count.restype = ctypes.c_ulonglong
         L.nuna_status_string.argtypes = [ctypes.c_int]
@@ -159,6 +194,43 @@ def nuna_chain_launch(chain, stream=None, check=True) -> int:
 
 def nuna_chain_destroy(chain) -> int:
     return lib().nuna_chain_destroy(chain)
+
+
+def nuna_probe_topology(bufs, nbytes=None, stream=None, check=True):
+    """Probes the given device buffers; returns a ``NunaTopology`` (or the status when check=False fails)."""
+    if nbytes is None:
+        nbytes = [b.numel() * b.element_size() for b in bufs]
+    sizes = (ctypes.c_size_t * len(bufs))(*[int(x) for x in nbytes])
+    topo = NunaTopology()
+    st = lib().nuna_probe_topology(ptr_table(bufs), sizes, len(bufs), ctypes.byref(topo), _stream(stream))
+    _finish(st, "nuna_probe_topology", check)
+    return topo if st == NUNA_OK else st
+
+
+def debug_analyse_topology(lat, lat_rep):
+    """Host-side clustering / verdict on a caller-supplied (num_sms x num_lines) float32 latency matrix."""
+    import numpy as np
+    a = np.ascontiguousarray(lat, dtype=np.float32)
+    b = np.ascontiguousarray(lat_rep, dtype=np.float32)
+    topo = NunaTopology()
+    fp = ctypes.POINTER(ctypes.c_float)
+    st = lib().nuna_debug_analyse_topology(a.ctypes.data_as(fp), b.ctypes.data_as(fp), a.shape[0], a.shape[1],
+                                           ctypes.byref(topo))
+    if st != NUNA_OK:
+        raise NunaError(st, "nuna_debug_analyse_topology")
+    return topo
+
+
+def debug_chain(nnodes: int, seed: int, start: int, steps: int):
+    """The probe's single-cycle permutation and the node a host walk of `steps` steps ends on."""
+    import numpy as np
+    nxt = np.zeros(nnodes, dtype=np.uint32)
+    end = ctypes.c_uint(0)
+    st = lib().nuna_debug_chain(nxt.ctypes.data_as(ctypes.POINTER(ctypes.c_uint)), nnodes, seed, start, steps,
+                                ctypes.byref(end))
+    if st != NUNA_OK:
+        raise NunaError(st, "nuna_debug_chain")
+    return nxt, end.value
 
 
 def nuna_device_status() -> int:

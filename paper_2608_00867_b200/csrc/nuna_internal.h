@@ -27,6 +27,8 @@ struct Context {
     int unroll_override = 0;             // NUNA_UNROLL
     int coloc_override = 0;              // NUNA_COLOC: destinations of a tile per block (2, 4, 8)
     size_t auto_min_bytes = 0;           // NUNA_PLACE_AUTO picks the aware kernel from this size per rank
+    nuna_topology_t topology = {};       // last probe result (have_topology says whether it is valid)
+    bool have_topology = false;
     std::mutex mutex;
 };
 
