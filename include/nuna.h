@@ -159,6 +159,29 @@ int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks,
 int nuna_allgather(const void* const* src, void* const* dst, int nranks,
                    size_t shard_count, int dtype, unsigned flags, void* stream);
 
+/* Two-shot allreduce for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this is a deployment convenience of the library.)  Some hosts of this code cannot call cudaMalloc
+ * on the request path: an inference server that has handed the whole GPU to its own memory pool, where
+ * a raw allocation can fail or fragment the pool, or a latency-critical loop that cannot afford the
+ * device-wide synchronisation and the failure modes an allocation brings.  This entry point computes
+ * exactly what nuna_allreduce_twoshot computes (flag-barrier form, same bits) but takes its shard
+ * intermediate and its barrier words from a fixed array compiled into the library, so it never calls
+ * cudaMalloc, cudaFree or any allocating routine, and it does not create the per-device context.
+ *  - Limit: count <= NUNA_STATIC_MAX_COUNT elements per rank (4 MiB of bf16); larger counts return
+ *    NUNA_ERR_TOO_LARGE and print the limit.  The array costs 4 MiB of device memory on every GPU
+ *    that loads the library, for the life of the process.
+ *  - The first call on a device looks up the array's device address and zeroes the barrier words
+ *    (a synchronous 16-byte cudaMemset); make that first call before starting any stream capture.
+ *  - All calls on a device share the one array, which keeps the previous call's shard; the kernel
+ *    overwrites every element it later reads, so stale contents never reach a result.  Two calls that
+ *    overlap on the GPU (different streams, no ordering) race on it: keep calls stream-ordered.
+ *  - A barrier that times out (1 s) latches NUNA_ERR_TIMEOUT in the array's own status word, which
+ *    this entry point does not expose; results are then undefined.  src / dst / nranks / dtype /
+ *    stream and the argument errors are those of nuna_allreduce_twoshot; there is no flags word.      */
+#define NUNA_STATIC_MAX_COUNT (2 * 1024 * 1024)
+int nuna_allreduce_twoshot_static(const void* const* src, void* const* dst, int nranks,
+                                  size_t count, int dtype, void* stream);
+
 /* End-to-end variant with HOST buffers: src[r] / dst[d] are HOST pointers to `count` elements (pinned
  * or pageable).  Copies the sources to library-owned device staging buffers, runs the one-shot
  * (two_shot == 0) or two-shot allreduce, copies every destination back and synchronises.  Allocates

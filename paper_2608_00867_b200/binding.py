@@ -76,6 +76,8 @@ def lib() -> ctypes.CDLL:
         for name in ("nuna_allreduce_oneshot", "nuna_allreduce_twoshot", "nuna_reduce_scatter", "nuna_allgather"):
             getattr(L, name).argtypes = coll
             getattr(L, name).restype = ctypes.c_int
+        L.nuna_allreduce_twoshot_static.argtypes = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_void_p]
+        L.nuna_allreduce_twoshot_static.restype = ctypes.c_int
         L.nuna_allreduce_host.argtypes = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint, ctypes.c_int]
         L.nuna_allreduce_host.restype = ctypes.c_int
         L.nuna_init.argtypes = [ctypes.c_size_t]
@@ -162,6 +164,16 @@ def nuna_reduce_scatter(src, dst, shard_count, dtype=NUNA_BF16, flags=0, stream=
 
 def nuna_allgather(src, dst, shard_count, dtype=NUNA_BF16, flags=0, stream=None, check=True, nranks=None) -> int:
     return _collective("nuna_allgather", src, dst, shard_count, dtype, flags, stream, check, nranks)
+
+
+NUNA_STATIC_MAX_COUNT = 2 * 1024 * 1024
+
+
+def nuna_allreduce_twoshot_static(src, dst, count, dtype=NUNA_BF16, stream=None, check=True) -> int:
+    """The two-shot allreduce that never allocates: its scratch is a fixed array inside the library
+    (at most NUNA_STATIC_MAX_COUNT elements per rank).  For callers that cannot call cudaMalloc."""
+    st = lib().nuna_allreduce_twoshot_static(ptr_table(src), ptr_table(dst), len(src), count, dtype, _stream(stream))
+    return _finish(st, "nuna_allreduce_twoshot_static", check)
 
 
 def nuna_allreduce_host(src, dst, count, dtype=NUNA_BF16, flags=0, two_shot=False, check=True) -> int:

@@ -524,3 +524,79 @@ int nuna_debug_barrier_selftest(unsigned grid, unsigned expected, unsigned timeo
 }
 
 }  // extern "C"
+
+// ---- two-shot allreduce for callers that cannot allocate ------------------------------------------
+//
+// Everything the flag-barrier two-shot needs beyond its inputs and outputs -- the shard
+// intermediate and the barrier words -- lives in the two file-scope device arrays below, which
+// every GPU that loads this library carries from module load to process exit (4 MiB + 16 bytes).
+// In host code the names `g_static_shard` and `g_static_barrier` are only stand-ins for the
+// symbols, not device addresses; the addresses a kernel can use come from cudaGetSymbolAddress,
+// looked up once per device, with that device current, on the entry point's first call there.
+namespace nuna {
+
+static __device__ __align__(256) unsigned char g_static_shard[NUNA_STATIC_MAX_COUNT * 2];
+static __device__ __align__(256) BarrierWords g_static_barrier;
+
+struct StaticSetup {
+    bool ready = false;
+    uint4* shard = nullptr;              // device address of g_static_shard on this device
+    BarrierWords* barrier = nullptr;     // device address of g_static_barrier on this device
+    int num_sms = 0;
+};
+static StaticSetup g_static_setup[kMaxDevices];
+static std::mutex g_static_mutex;
+
+// Once per device: resolve the two symbols and zero the barrier words.  No allocation.
+static int static_setup(StaticSetup** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return NUNA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticSetup& s = g_static_setup[dev];
+    if (!s.ready) {
+        void* shard = nullptr;
+        void* barrier = nullptr;
+        if (cudaGetSymbolAddress(&shard, g_static_shard) != cudaSuccess || !shard) return NUNA_ERR_CUDA;
+        if (cudaGetSymbolAddress(&barrier, g_static_barrier) != cudaSuccess || !barrier) return NUNA_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&s.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || s.num_sms < 1)
+            return NUNA_ERR_CUDA;
+        // the barrier counts arrivals from zero; the shard needs no clearing (written before it is read)
+        if (cudaMemset(barrier, 0, sizeof(BarrierWords)) != cudaSuccess) return NUNA_ERR_CUDA;
+        s.shard = static_cast<uint4*>(shard);
+        s.barrier = static_cast<BarrierWords*>(barrier);
+        s.ready = true;
+    }
+    *out = &s;
+    return NUNA_OK;
+}
+
+}  // namespace nuna
+
+extern "C" int nuna_allreduce_twoshot_static(const void* const* src, void* const* dst, int nranks, size_t count,
+                                             int dtype, void* stream)
+{
+    int st = check_args(src, dst, nranks, count, count, dtype, 0u, true);
+    if (st != NUNA_OK || count == 0) return st;
+    if (count > (size_t)NUNA_STATIC_MAX_COUNT) {
+        fprintf(stderr, "nuna_allreduce_twoshot_static: count %zu exceeds NUNA_STATIC_MAX_COUNT (%d elements); "
+                        "use nuna_allreduce_twoshot for larger messages\n", count, (int)NUNA_STATIC_MAX_COUNT);
+        return NUNA_ERR_TOO_LARGE;
+    }
+    StaticSetup* s = nullptr;
+    if ((st = static_setup(&s)) != NUNA_OK) return st;
+    const RankPtrs p = make_ptrs(src, dst, nranks);
+    const size_t chunk_vec = ceil_div(ceil_div(count, (size_t)nranks), (size_t)kVecElems);
+    const int u = nranks >= 8 ? 1 : nranks >= 4 ? 2 : 4;
+    return dispatch(nranks, u, [&](auto n_, auto u_) -> int {
+        NUNA_NU(n_, u_);
+        static int occ = 0;
+        auto k = k_twoshot_fused<N, U>;
+        const size_t tiles_per_chunk = ceil_div(chunk_vec, (size_t)kThreads * U);
+        const size_t cap = (size_t)s->num_sms * (size_t)occupancy(nullptr, k, &occ);   // all blocks co-resident
+        const unsigned grid = (unsigned)std::max<size_t>(1, std::min(tiles_per_chunk * N, cap));
+        return launch(k, grid, (cudaStream_t)stream, kLaunchCooperative, p, s->shard, count, chunk_vec, s->barrier,
+                      1000000000ull);
+    });
+}
+
