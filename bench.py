@@ -265,6 +265,16 @@ def run_gpu(args):
     floor_pdl_us = per_call_us(lambda s, d, st: nb.nuna_launch_floor(grid_blocks, flags=nb.NUNA_LAUNCH_PDL, stream=st), sets, 1000, 3)
 
     extras = {}
+    # ---- placement on the headline workload: round-robin baseline vs the two placement-aware kernels ---------
+    # (per-SM work lists use the topology of a probe run here on the first buffer set)
+    nb.nuna_probe_topology(list(sets[0][0]) + list(sets[0][1]))
+    place = {}
+    for pname, pflags in (("roundrobin", nb.NUNA_PLACE_ROUNDROBIN), ("aware_colocated", nb.NUNA_PLACE_AWARE),
+                          ("aware_sm_lists", nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS)):
+        fn = lambda s, d, st, f=pflags: nb.nuna_allreduce_oneshot(s, d, count, flags=f, stream=st)
+        place[pname] = {"cold_us": round(per_call_us(fn, sets, 1000, 3), 3),
+                        "l2_resident_us": round(per_call_us(fn, sets[:1], 1000, 3), 3)}
+    extras["placement_512KiB"] = place
     if True:
         # ---- end to end through the host-buffer entry point (pinned host memory) -----------------------
         hsrc = [torch.from_numpy(a.view(np.int16).copy()).pin_memory() for a in workloads.make(w)]
@@ -325,6 +335,7 @@ def run_gpu(args):
             "roundrobin_pdl": nb.NUNA_PLACE_ROUNDROBIN | nb.NUNA_LAUNCH_PDL,
             "aware_pdl": nb.NUNA_PLACE_AWARE | nb.NUNA_LAUNCH_PDL,
             "auto_resident_pdl": nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT | nb.NUNA_LAUNCH_PDL,
+            "aware_sm_lists_pdl": nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS | nb.NUNA_LAUNCH_PDL,
         }
         for tokens in workloads.CHAIN_TOKENS:
             wc = workloads.config_decode_chain(tokens)
@@ -425,6 +436,7 @@ def run_case(args):
     call = {
         "oneshot": lambda s, d: nb.nuna_allreduce_oneshot(s, d, count),
         "oneshot_aware": lambda s, d: nb.nuna_allreduce_oneshot(s, d, count, flags=nb.NUNA_PLACE_AWARE),
+        "oneshot_sm": lambda s, d: nb.nuna_allreduce_oneshot(s, d, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS),
         "twoshot": lambda s, d: nb.nuna_allreduce_twoshot(s, d, count),
         "twoshot_put": lambda s, d: nb.nuna_allreduce_twoshot(s, d, count, flags=nb.NUNA_TWOSHOT_PUT),
         "allgather": lambda s, d: nb.nuna_allgather(s, d, count),
@@ -448,7 +460,7 @@ def main():
     ap.add_argument("--sweep-max", type=int, default=26)
     ap.add_argument("--case", default=None,
                     help="ALGO:LOG2BYTES[:LAUNCHES] -- run a few eager launches of one algorithm at one size and "
-                         "exit (for ncu captures); ALGO in oneshot, oneshot_aware, twoshot, twoshot_put, allgather")
+                         "exit (for ncu captures); ALGO in oneshot, oneshot_aware, oneshot_sm, twoshot, twoshot_put, allgather")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

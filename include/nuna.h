@@ -79,6 +79,13 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* on
  * its first global access, so results are those of an ordinary stream-ordered launch.  Ignored by the
  * flag-barrier two-shot (a cooperative launch) and above 16 MiB of sources, where it does not pay.     */
 #define NUNA_LAUNCH_PDL       64u
+/* `flags`, bit 7, with NUNA_PLACE_AWARE on nuna_allreduce_oneshot: dispatch the co-located groups through
+ * per-SM work lists.  The lists are planned by Algorithm 1 from the topology the last
+ * nuna_probe_topology call on this device found (none: one domain, SMs in index order); persistent blocks
+ * read %smid, claim the groups planned for their SM and then take over what is left elsewhere.  The
+ * first call for a given (nranks, count) builds and uploads the plan (allocates: NUNA_ERR_CAPTURING on a
+ * capturing stream); later calls only launch.  Calls sharing a plan must be stream-ordered.             */
+#define NUNA_PLACE_SM_LISTS   128u
 
 /* ---- topology probe --------------------------------------------------------------------------------
  * Result of nuna_probe_topology: caller-owned, plain data, fixed maximum sizes.  Latencies are in SM
@@ -127,6 +134,38 @@ typedef struct nuna_topology {
  * stream.  Latency values are hardware facts and carry no parity claim.                               */
 int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
                         nuna_topology_t* out, void* stream);
+
+/* ---- placement planner (host only; no CUDA call) ----------------------------------------------------
+ * The paper's Algorithm 1 (Section 4.2): logical allocation of thread blocks and the chunks they touch
+ * into groups, groups dealt round-robin to nar_max domains, then per block the first compute unit of
+ * its domain with budget left and a memory stack near it.  Chunks -- the paper's
+ * (chunk_id, buffer_type, gpu_id) tuples -- are numbered 0..num_chunks-1 by the caller.
+ * Conventions where the text leaves a choice: first group -> domain 0; a block joins the group owning
+ * most of its chunks, ties to the group created first; owned chunks stay where they are; groups sorted
+ * by decreasing chunk bytes, stable; no CU with budget -> the CU of the domain with most budget left;
+ * stack preference = the CU's nearest stack, then the others in increasing index; a chunk keeps the
+ * first stack it was given.  Budgets are counted per (gpu, CU) and per (gpu, stack), in bytes.          */
+typedef struct nuna_plan_input {
+    int num_tbs;                 /* |W|                                                                    */
+    const int* tb_gpu;           /* [num_tbs] gpu of each thread block                                      */
+    const int* tb_chunk_begin;   /* [num_tbs + 1] CSR offsets into tb_chunks                                */
+    const int* tb_chunks;        /* chunk ids touched by each block (C_tb)                                  */
+    int num_chunks;
+    const long long* chunk_bytes;/* [num_chunks]                                                            */
+    int num_cus;
+    const int* cu_domain;        /* [num_cus] domain of each compute unit, 0..nar_max-1                     */
+    const int* cu_rank;          /* [num_cus] preference inside the domain, lower = nearer (ties: CU index) */
+    int num_stacks;
+    const int* cu_stack;         /* [num_cus] nearest memory stack                                          */
+    long long r_max_cu;          /* budget per compute unit, bytes                                          */
+    long long r_max_stack;       /* budget per memory stack, bytes                                          */
+    int nar_max;                 /* number of domains                                                       */
+} nuna_plan_input_t;
+
+/* Outputs, caller-allocated: m_compute[num_tbs] (CU per block); optional (may be NULL):
+ * m_memory[num_chunks] (stack per chunk, -1 if untouched), tb_domain[num_tbs], tb_group[num_tbs]
+ * (index of the block's group in placement order).  Returns NUNA_ERR_INVALID_ARG on malformed input.   */
+int nuna_plan_placement(const nuna_plan_input_t* in, int* m_compute, int* m_memory, int* tb_domain, int* tb_group);
 
 /* Create the calling thread's current device's context (flag-barrier words, status word, work cursors,
  * two-shot shard scratch of `scratch_bytes`).  Called implicitly by the first collective on a device;

@@ -26,6 +26,7 @@ NUNA_PLACE_ROUNDROBIN, NUNA_PLACE_AWARE, NUNA_PLACE_AUTO = 0, 1, 2
 NUNA_TWOSHOT_PUT = 16
 NUNA_HINT_RESIDENT = 32
 NUNA_LAUNCH_PDL = 64
+NUNA_PLACE_SM_LISTS = 128
 
 NUNA_MAX_SMS, NUNA_MAX_PROBE_BUFS, NUNA_PROBE_REGIONS, NUNA_MAX_PROBE_LINES = 256, 32, 8, 2048
 NUNA_TOPO_UNIFORM, NUNA_TOPO_NONUNIFORM = 0, 1
@@ -50,6 +51,18 @@ class NunaTopology(ctypes.Structure):
         ("line_buf", ctypes.c_ubyte * NUNA_MAX_PROBE_LINES),
         ("line_region", ctypes.c_ubyte * NUNA_MAX_PROBE_LINES),
         ("line_home", ctypes.c_ubyte * NUNA_MAX_PROBE_LINES),
+    ]
+
+
+class NunaPlanInput(ctypes.Structure):
+    """Mirror of ``nuna_plan_input_t`` (include/nuna.h)."""
+    _ip, _lp = ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_longlong)
+    _fields_ = [
+        ("num_tbs", ctypes.c_int), ("tb_gpu", _ip), ("tb_chunk_begin", _ip), ("tb_chunks", _ip),
+        ("num_chunks", ctypes.c_int), ("chunk_bytes", _lp),
+        ("num_cus", ctypes.c_int), ("cu_domain", _ip), ("cu_rank", _ip),
+        ("num_stacks", ctypes.c_int), ("cu_stack", _ip),
+        ("r_max_cu", ctypes.c_longlong), ("r_max_stack", ctypes.c_longlong), ("nar_max", ctypes.c_int),
     ]
 
 
@@ -102,6 +115,13 @@ def lib() -> ctypes.CDLL:
         L.nuna_debug_chain.argtypes = [ctypes.POINTER(ctypes.c_uint), ctypes.c_int, ctypes.c_ulonglong, ctypes.c_uint,
                                        ctypes.c_int, ctypes.POINTER(ctypes.c_uint)]
         L.nuna_debug_chain.restype = ctypes.c_int
+        up = ctypes.POINTER(ctypes.c_uint)
+        L.nuna_debug_plan_oneshot.argtypes = [ctypes.POINTER(NunaTopology), ctypes.c_int, ctypes.c_int, ctypes.c_size_t,
+                                              ctypes.c_size_t, ctypes.c_int, up, up]
+        L.nuna_debug_plan_oneshot.restype = ctypes.c_int
+        ip = ctypes.POINTER(ctypes.c_int)
+        L.nuna_plan_placement.argtypes = [ctypes.POINTER(NunaPlanInput), ip, ip, ip, ip]
+        L.nuna_plan_placement.restype = ctypes.c_int
         L.nuna_launch_count.argtypes = []
         L.nuna_launch_count.restype = ctypes.c_ulonglong
         L.nuna_status_string.argtypes = [ctypes.c_int]
@@ -233,6 +253,19 @@ def debug_analyse_topology(lat, lat_rep):
     return topo
 
 
+def debug_plan_oneshot(topo, num_sms: int, nranks: int, ntiles: int, tile_bytes: int, generic: bool):
+    """Per-SM work lists planned for a one-shot: returns a list (one entry per SM) of tile lists."""
+    import numpy as np
+    off = np.zeros(num_sms + 1, dtype=np.uint32)
+    tiles = np.zeros(max(ntiles, 1), dtype=np.uint32)
+    up = ctypes.POINTER(ctypes.c_uint)
+    st = lib().nuna_debug_plan_oneshot(ctypes.byref(topo) if topo is not None else None, num_sms, nranks, ntiles,
+                                       tile_bytes, 1 if generic else 0, off.ctypes.data_as(up), tiles.ctypes.data_as(up))
+    if st != NUNA_OK:
+        raise NunaError(st, "nuna_debug_plan_oneshot")
+    return [tiles[off[s]:off[s + 1]].tolist() for s in range(num_sms)]
+
+
 def debug_chain(nnodes: int, seed: int, start: int, steps: int):
     """The probe's single-cycle permutation and the node a host walk of `steps` steps ends on."""
     import numpy as np
@@ -243,6 +276,39 @@ def debug_chain(nnodes: int, seed: int, start: int, steps: int):
     if st != NUNA_OK:
         raise NunaError(st, "nuna_debug_chain")
     return nxt, end.value
+
+
+def nuna_plan_placement(tb_gpu, tb_chunks, chunk_bytes, cu_domain, cu_rank, cu_stack, num_stacks,
+                        r_max_cu, r_max_stack, nar_max, check=True):
+    """Algorithm 1 on the host.  ``tb_chunks``: one list of chunk ids per thread block.
+    Returns (m_compute, m_memory, tb_domain, tb_group) as lists."""
+    import numpy as np
+    T, C, U = len(tb_gpu), len(chunk_bytes), len(cu_domain)
+    begin = np.zeros(T + 1, dtype=np.int32)
+    for t, cs in enumerate(tb_chunks):
+        begin[t + 1] = begin[t] + len(cs)
+    flat = np.array([c for cs in tb_chunks for c in cs] or [0], dtype=np.int32)
+    arrs = {
+        "tb_gpu": np.array(list(tb_gpu) or [0], dtype=np.int32), "begin": begin, "flat": flat,
+        "bytes": np.array(list(chunk_bytes) or [0], dtype=np.int64),
+        "dom": np.array(cu_domain, dtype=np.int32), "rank": np.array(cu_rank, dtype=np.int32),
+        "stack": np.array(cu_stack, dtype=np.int32),
+    }
+    ip, lp = ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_longlong)
+    inp = NunaPlanInput(T, arrs["tb_gpu"].ctypes.data_as(ip), arrs["begin"].ctypes.data_as(ip),
+                        arrs["flat"].ctypes.data_as(ip), C, arrs["bytes"].ctypes.data_as(lp), U,
+                        arrs["dom"].ctypes.data_as(ip), arrs["rank"].ctypes.data_as(ip), num_stacks,
+                        arrs["stack"].ctypes.data_as(ip), r_max_cu, r_max_stack, nar_max)
+    mc = np.full(max(T, 1), -1, dtype=np.int32)
+    mm = np.full(max(C, 1), -1, dtype=np.int32)
+    td = np.full(max(T, 1), -1, dtype=np.int32)
+    tg = np.full(max(T, 1), -1, dtype=np.int32)
+    st = lib().nuna_plan_placement(ctypes.byref(inp), mc.ctypes.data_as(ip), mm.ctypes.data_as(ip),
+                                   td.ctypes.data_as(ip), tg.ctypes.data_as(ip))
+    _finish(st, "nuna_plan_placement", check)
+    if st != NUNA_OK:
+        return st
+    return mc[:T].tolist(), mm[:C].tolist(), td[:T].tolist(), tg[:T].tolist()
 
 
 def nuna_device_status() -> int:

@@ -9,6 +9,7 @@
 #include <cstring>
 #include <mutex>
 #include <type_traits>
+#include <vector>
 
 namespace nuna {
 
@@ -80,7 +81,7 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
     if (nranks < 1) return NUNA_ERR_INVALID_ARG;
     if (dtype != NUNA_BF16) return (dtype == NUNA_F16 || dtype == NUNA_F32) ? NUNA_ERR_UNSUPPORTED_DTYPE
                                                                              : NUNA_ERR_UNSUPPORTED_DTYPE;
-    if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT | NUNA_HINT_RESIDENT | NUNA_LAUNCH_PDL)) != 0u ||
+    if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT | NUNA_HINT_RESIDENT | NUNA_LAUNCH_PDL | NUNA_PLACE_SM_LISTS)) != 0u ||
         (flags & NUNA_PLACE_MASK) == 3u)
         return NUNA_ERR_INVALID_ARG;
     if (src_elems > ((size_t)1 << 40) || dst_elems > ((size_t)1 << 40)) return NUNA_ERR_TOO_LARGE;
@@ -226,6 +227,162 @@ static bool aware_pays_off(const Context* c, int nranks, size_t count, unsigned 
 }
 
 
+// ---- per-SM work lists for the one-shot (Algorithm 1 applied to its regular workload) ----------------
+//
+// Thread blocks = work items (tile, d); item (t, d) touches the N source chunks of tile t and the
+// destination chunk (d, t).  Domains and the order of SMs inside a domain come from the probe
+// (nearest = lowest mean hit latency).  The per-SM budget R_max is ceil(groups per domain / SMs of
+// the smallest domain) whole groups, so a small workload fills only the nearest SMs, one group each,
+// and a large one spreads evenly.  Up to kGenericPlanTiles tiles the lists are produced by the
+// general planner (nuna_plan_placement); beyond that by the closed form it reduces to for this
+// workload (tile t -> domain t mod D, SMs of the domain filled in preference order), which the host
+// tests check against the general planner.
+constexpr size_t kGenericPlanTiles = 1024;
+
+void plan_oneshot_lists(const nuna_topology_t* topo, int num_sms, int nranks, size_t ntiles, size_t tile_bytes,
+                        bool generic, std::vector<std::vector<unsigned>>& lists)
+{
+    lists.assign((size_t)num_sms, {});
+    const bool split = topo && topo->verdict == NUNA_TOPO_NONUNIFORM && topo->num_domains == 2;
+    const int D = split ? 2 : 1;
+    std::vector<int> dom(num_sms, 0), rank(num_sms, 0), order(num_sms);
+    for (int s = 0; s < num_sms; ++s) {
+        order[s] = s;
+        if (split && s < NUNA_MAX_SMS) dom[s] = topo->sm_domain[s];
+    }
+    if (topo && topo->sms_reported > 0)
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+            const float la = a < NUNA_MAX_SMS ? topo->sm_lat_hit[a] : 0.f, lb = b < NUNA_MAX_SMS ? topo->sm_lat_hit[b] : 0.f;
+            return la < lb;
+        });
+    for (int i = 0; i < num_sms; ++i) rank[order[i]] = i;
+    int smallest = num_sms;
+    if (split) {
+        int n1 = 0;
+        for (int s = 0; s < num_sms; ++s) n1 += dom[s];
+        smallest = std::max(1, std::min(n1, num_sms - n1));
+    }
+    const size_t per_domain = ceil_div(ntiles, (size_t)D);
+    const size_t budget = std::max<size_t>(1, ceil_div(per_domain, (size_t)smallest));        // groups per SM
+    if (generic) {
+        const int N = nranks;
+        std::vector<int> tb_gpu(ntiles * N, 0), begin(ntiles * N + 1, 0), chunks;
+        chunks.reserve(ntiles * N * (N + 1));
+        for (size_t t = 0; t < ntiles; ++t)
+            for (int d = 0; d < N; ++d) {
+                for (int r = 0; r < N; ++r) chunks.push_back((int)(r * ntiles + t));
+                chunks.push_back((int)((N + d) * ntiles + t));
+                begin[t * N + d + 1] = (int)chunks.size();
+            }
+        std::vector<long long> cbytes(2 * (size_t)N * ntiles, (long long)tile_bytes);
+        std::vector<int> stack(num_sms, 0), m_compute(ntiles * N, -1);
+        nuna_plan_input_t in = {};
+        in.num_tbs = (int)(ntiles * N); in.tb_gpu = tb_gpu.data(); in.tb_chunk_begin = begin.data(); in.tb_chunks = chunks.data();
+        in.num_chunks = (int)cbytes.size(); in.chunk_bytes = cbytes.data();
+        in.num_cus = num_sms; in.cu_domain = dom.data(); in.cu_rank = rank.data();
+        in.num_stacks = 1; in.cu_stack = stack.data();
+        in.r_max_cu = (long long)(budget * (size_t)N * (size_t)(N + 1) * tile_bytes);
+        in.r_max_stack = (long long)1 << 60;
+        in.nar_max = D;
+        if (nuna_plan_placement(&in, m_compute.data(), nullptr, nullptr, nullptr) == NUNA_OK) {
+            for (size_t t = 0; t < ntiles; ++t) lists[(size_t)m_compute[t * N]].push_back((unsigned)t);
+            return;
+        }
+        lists.assign((size_t)num_sms, {});
+    }
+    // closed form
+    std::vector<std::vector<int>> dom_sms(D);
+    for (int i = 0; i < num_sms; ++i) dom_sms[dom[order[i]]].push_back(order[i]);
+    std::vector<size_t> used(D, 0);
+    for (size_t t = 0; t < ntiles; ++t) {
+        const int d = (int)(t % (size_t)D);
+        size_t slot = used[d]++ / budget;
+        if (slot >= dom_sms[d].size()) slot = dom_sms[d].size() - 1;      // cannot happen with the budget above
+        lists[(size_t)dom_sms[d][slot]].push_back((unsigned)t);
+    }
+}
+
+static int get_sm_plan(Context* c, int nranks, size_t count, int coloc, cudaStream_t stream, SmPlan** out)
+{
+    std::lock_guard<std::mutex> lock(c->mutex);
+    const auto key = std::make_tuple(nranks, count, coloc);
+    auto it = c->sm_plans.find(key);
+    if (it == c->sm_plans.end()) {
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone)
+            return NUNA_ERR_CAPTURING;                 // building a plan allocates: make one plain call first
+        const size_t lanes = (size_t)(kThreads / coloc);
+        const size_t ntiles = ceil_div(count / kVecElems, lanes);
+        std::vector<std::vector<unsigned>> lists;
+        plan_oneshot_lists(c->have_topology ? &c->topology : nullptr, c->num_sms, nranks, ntiles, lanes * 16,
+                           ntiles <= kGenericPlanTiles, lists);
+        std::vector<unsigned> off((size_t)c->num_sms + 1, 0), tiles;
+        tiles.reserve(ntiles);
+        for (int s = 0; s < c->num_sms; ++s) {
+            tiles.insert(tiles.end(), lists[s].begin(), lists[s].end());
+            off[s + 1] = (unsigned)tiles.size();
+        }
+        SmPlan pl;
+        pl.total = (unsigned)tiles.size();
+        const size_t words = off.size() + std::max<size_t>(tiles.size(), 1) + 2 * (size_t)c->num_sms + 2;
+        unsigned* d = nullptr;
+        if (cudaMalloc(&d, words * sizeof(unsigned)) != cudaSuccess) return NUNA_ERR_CUDA;
+        std::vector<unsigned> host(words, 0u);
+        std::copy(off.begin(), off.end(), host.begin());
+        std::copy(tiles.begin(), tiles.end(), host.begin() + off.size());
+        const size_t cur0 = off.size() + std::max<size_t>(tiles.size(), 1);
+        pl.nonempty = 0;
+        for (int s = 0; s < c->num_sms; ++s) pl.nonempty += !lists[s].empty();
+        if (cudaMemcpy(d, host.data(), words * sizeof(unsigned), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaFree(d);
+            return NUNA_ERR_CUDA;
+        }
+        pl.base = d;
+        pl.off = d;
+        pl.tiles = d + off.size();
+        pl.cursor = d + cur0;
+        pl.present = d + cur0 + c->num_sms;
+        pl.ctl = d + cur0 + 2 * (size_t)c->num_sms;
+        it = c->sm_plans.emplace(key, pl).first;
+    }
+    *out = &it->second;
+    return NUNA_OK;
+}
+
+static int coloc_for(const Context* c, int nranks)
+{
+    int coloc = c->coloc_override > 0 ? c->coloc_override : 8;
+    while (coloc > 1 && coloc / 2 >= nranks) coloc >>= 1;
+    return coloc >= 8 ? 8 : coloc >= 4 ? 4 : 2;
+}
+
+// Everything a later launch of this shape would have to allocate (called before stream capture).
+int prepare_oneshot(Context* c, int nranks, size_t count, unsigned flags)
+{
+    if ((flags & NUNA_PLACE_MASK) == NUNA_PLACE_AWARE && (flags & NUNA_PLACE_SM_LISTS)) {
+        SmPlan* pl = nullptr;
+        return get_sm_plan(c, nranks, count, coloc_for(c, nranks), (cudaStream_t)0, &pl);
+    }
+    return NUNA_OK;
+}
+
+template <int N, int C>
+static int launch_sm_lists(Context* c, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
+{
+    static int occ = 0;
+    auto k = k_oneshot_sm<N, C>;
+    SmPlan* pl = nullptr;
+    const int st = get_sm_plan(c, N, count, C, stream, &pl);
+    if (st != NUNA_OK) return st;
+    SmLists sl;
+    sl.off = pl->off; sl.tiles = pl->tiles; sl.cursor = pl->cursor; sl.present = pl->present; sl.ctl = pl->ctl;
+    sl.nonempty = pl->nonempty; sl.num_sms = c->num_sms;
+    const size_t cap = (size_t)c->num_sms * (size_t)occupancy(c, k, &occ);
+    const unsigned grid = (unsigned)std::min(cap, std::max<size_t>((size_t)c->num_sms, (size_t)pl->total));
+    const unsigned blocks_per_sm = (unsigned)std::max<size_t>(1, grid / (size_t)c->num_sms);
+    return launch(k, grid, stream, mode, p, count, sl, blocks_per_sm);
+}
+
 template <int N, int C>
 static int launch_group(Context* c, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
 {
@@ -245,8 +402,15 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsi
     const unsigned place = flags & NUNA_PLACE_MASK;
     if (place == NUNA_PLACE_AWARE || (place == NUNA_PLACE_AUTO && aware_pays_off(c, nranks, count, flags))) {
         // co-location factor: C destinations of a tile share a block (C <= N rounded up to a power of two)
-        int coloc = c->coloc_override > 0 ? c->coloc_override : 8;
-        while (coloc > 1 && coloc / 2 >= nranks) coloc >>= 1;
+        const int coloc = coloc_for(c, nranks);
+        if (flags & NUNA_PLACE_SM_LISTS) {
+            return dispatch(nranks, 1, [&](auto n_, auto) -> int {
+                constexpr int N = decltype(n_)::value;
+                if (coloc >= 8) return launch_sm_lists<N, 8>(c, p, count, mode, stream);
+                if (coloc >= 4) return launch_sm_lists<N, 4>(c, p, count, mode, stream);
+                return launch_sm_lists<N, 2>(c, p, count, mode, stream);
+            });
+        }
         return dispatch(nranks, 1, [&](auto n_, auto) -> int {
             constexpr int N = decltype(n_)::value;
             if (coloc >= 8) return launch_group<N, 8>(c, p, count, mode, stream);
@@ -497,9 +661,27 @@ int nuna_shutdown(void)
     if (c->scratch) cudaFree(c->scratch);
     if (c->staging) cudaFree(c->staging);
     if (c->stream) cudaStreamDestroy(c->stream);
+    for (auto& kv : c->sm_plans) cudaFree(kv.second.base);
     delete c;
     g_ctx[dev] = nullptr;
     return NUNA_OK;
+}
+
+/* Test hook: the per-SM work lists planned for a one-shot of `ntiles` tiles under `topo` (NULL = no probe),
+ * by the general planner (generic != 0) or the closed form.  off: [num_sms + 1], tiles: [ntiles].          */
+int nuna_debug_plan_oneshot(const nuna_topology_t* topo, int num_sms, int nranks, size_t ntiles, size_t tile_bytes,
+                            int generic, unsigned* off, unsigned* tiles)
+{
+    if (num_sms < 1 || nranks < 1 || nranks > NUNA_MAX_RANKS || !off || !tiles) return NUNA_ERR_INVALID_ARG;
+    std::vector<std::vector<unsigned>> lists;
+    plan_oneshot_lists(topo, num_sms, nranks, ntiles, tile_bytes, generic != 0, lists);
+    size_t n = 0;
+    off[0] = 0;
+    for (int s = 0; s < num_sms; ++s) {
+        for (unsigned t : lists[s]) tiles[n++] = t;
+        off[s + 1] = (unsigned)n;
+    }
+    return n == ntiles ? NUNA_OK : NUNA_ERR_INVALID_ARG;
 }
 
 /* Test hook (not part of the public header): every block of a `grid`-block launch arrives at a flag

@@ -44,6 +44,7 @@ int nuna_chain_create(const void* const* src_sets, void* const* dst_sets, int ns
         std::lock_guard<std::mutex> lock(c->mutex);
         if ((st = ensure_scratch(c, (count * 2 + 15) & ~(size_t)15)) != NUNA_OK) return st;
     }
+    if (!two_shot && (st = prepare_oneshot(c, nranks, count, flags)) != NUNA_OK) return st;
     cudaStream_t cap = nullptr;
     if (cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking) != cudaSuccess) return NUNA_ERR_CUDA;
     cudaGraph_t graph = nullptr;

@@ -3,7 +3,10 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <map>
 #include <mutex>
+#include <tuple>
+#include <vector>
 
 #include "../../include/nuna.h"
 #include "nuna_types.h"
@@ -11,6 +14,18 @@
 namespace nuna {
 
 constexpr int kMaxDevices = 64;
+
+// Device-resident per-SM work lists of one (nranks, count, co-location) one-shot shape.
+struct SmPlan {
+    unsigned* base = nullptr;            // one allocation: off | tiles | cursor | present | ctl
+    unsigned* off = nullptr;
+    unsigned* tiles = nullptr;
+    unsigned* cursor = nullptr;
+    unsigned* present = nullptr;
+    unsigned* ctl = nullptr;
+    unsigned total = 0;
+    unsigned nonempty = 0;
+};
 
 struct Context {
     int device = -1;
@@ -29,6 +44,7 @@ struct Context {
     size_t auto_min_bytes = 0;           // NUNA_PLACE_AUTO picks the aware kernel from this size per rank
     nuna_topology_t topology = {};       // last probe result (have_topology says whether it is valid)
     bool have_topology = false;
+    std::map<std::tuple<int, size_t, int>, SmPlan> sm_plans;
     std::mutex mutex;
 };
 
@@ -38,6 +54,9 @@ int get_context(Context** out);
 int ensure_scratch(Context* c, size_t bytes);
 int check_args(const void* const* src, void* const* dst, int nranks, size_t src_elems, size_t dst_elems,
                int dtype, unsigned flags, bool device_ptrs);
+void plan_oneshot_lists(const nuna_topology_t* topo, int num_sms, int nranks, size_t ntiles, size_t tile_bytes,
+                        bool generic, std::vector<std::vector<unsigned>>& lists);
+int prepare_oneshot(Context* c, int nranks, size_t count, unsigned flags);
 int launch_oneshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream);
 int launch_twoshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream);
 int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shard, unsigned flags, cudaStream_t stream);

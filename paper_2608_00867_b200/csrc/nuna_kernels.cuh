@@ -245,6 +245,149 @@ k_oneshot_group(const RankPtrs p, const size_t count, const size_t ntiles)
     }
 }
 
+// ---- one-shot allreduce through per-SM work lists (the planner's M_compute at SM granularity) ------------
+//
+// CUDA has no thread-block -> SM affinity mask (the paper's dispatcher mechanism, Section 4.2.3), so
+// affinity is taken from the other end: a block reads %smid and claims, one group at a time, the
+// groups the planner put on that SM's list (an atomic cursor per SM, so two blocks that land on the
+// same SM share its list).  Each SM with a list records that a block arrived there.  A block that
+// runs out of work leaves once every list has such a block; if some list has none (the hardware
+// scheduler gave that SM no block) it adopts that list instead -- the paper's fall-back of ignoring
+// the affinity (Section 4.2.3).  Completion therefore never depends on where blocks land, and no
+// block ever waits for another.  The last block to finish rewinds all counters, which makes the
+// launch replayable from a CUDA graph without host work.
+struct SmLists {
+    const unsigned* off;        // [num_sms + 1] offsets into tiles
+    const unsigned* tiles;      // tile index of every planned group, grouped by SM
+    unsigned* cursor;           // [num_sms] next unclaimed entry of each SM's list
+    unsigned* present;          // [num_sms] non-zero once a block has arrived on that SM
+    unsigned* ctl;              // ctl[0]: non-empty lists whose SM has a block; ctl[1]: blocks that have left
+    unsigned nonempty;          // number of non-empty lists
+    int num_sms;
+};
+
+__device__ __forceinline__ unsigned read_smid_reg()
+{
+    unsigned s;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(s));
+    return s;
+}
+
+__device__ __forceinline__ unsigned ld_volatile_u32(const unsigned* p)
+{
+    unsigned v;
+    asm volatile("ld.volatile.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+constexpr unsigned kMaxBatch = 32;
+
+// Lane 0 claims up to `batch` entries of list v with one atomic add (the cursor may run past the end;
+// the last block rewinds it); the warp's lanes then fetch the claimed tile indices in one parallel
+// load.  `announce`: lane 1 records, in the same round trip, that SM v's list has a block serving it.
+// `exhausted` is set when the claim reached the end of the list.
+__device__ __forceinline__ unsigned claim_from(const SmLists& sl, unsigned v, unsigned len, unsigned batch, bool announce,
+                                               unsigned* sh_tiles, bool& exhausted)
+{
+    const unsigned lane = threadIdx.x & 31u;
+    unsigned j0 = 0u;
+    if (lane == 0 && len != 0u) j0 = atomicAdd(sl.cursor + v, batch);
+    if (lane == 1 && announce && len != 0u && atomicExch(sl.present + v, 1u) == 0u) atomicAdd(sl.ctl, 1u);
+    j0 = __shfl_sync(0xFFFFFFFFu, j0, 0);
+    const unsigned n = (len != 0u && j0 < len) ? min(batch, len - j0) : 0u;
+    exhausted = (len == 0u) || (j0 + batch >= len);
+    if (lane < n) sh_tiles[lane] = sl.tiles[sl.off[v] + j0 + lane];
+    return n;
+}
+
+// A list nobody is serving: its SM has no block (the hardware scheduler is free to do that).  Scans the
+// SMs 32 at a time and returns one such SM, or ~0u.
+__device__ __forceinline__ unsigned find_orphan(const SmLists& sl, unsigned own)
+{
+    const unsigned lane = threadIdx.x & 31u;
+    for (unsigned base = 0; base < (unsigned)sl.num_sms; base += 32u) {
+        const bool valid = base + lane < (unsigned)sl.num_sms;
+        const unsigned w = (own + 1u + base + lane) % (unsigned)sl.num_sms;
+        const unsigned wl = valid ? sl.off[w + 1] - sl.off[w] : 0u;
+        const bool orphan = wl != 0u && ld_volatile_u32(sl.present + w) == 0u && ld_volatile_u32(sl.cursor + w) < wl;
+        const unsigned mask = __ballot_sync(0xFFFFFFFFu, orphan);
+        if (mask != 0u) return __shfl_sync(0xFFFFFFFFu, w, __ffs(mask) - 1);
+    }
+    return 0xFFFFFFFFu;
+}
+
+template <int N, int C>
+__global__ void __launch_bounds__(kThreads, min_blocks(N))
+k_oneshot_sm(const RankPtrs p, const size_t count, const SmLists sl, const unsigned blocks_per_sm)
+{
+    pdl_wait();
+    constexpr int kSplit = (N + C - 1) / C;
+    __shared__ unsigned sh_n;
+    __shared__ unsigned sh_tiles[kMaxBatch];
+    const size_t nvec = count / kVecElems;
+    const unsigned own = read_smid_reg() % (unsigned)sl.num_sms;
+    const unsigned own_len = sl.off[own + 1] - sl.off[own];
+    // an SM's list is shared by the blocks resident there: one claim per block takes its whole share
+    const unsigned batch = min(kMaxBatch, max(1u, (own_len + blocks_per_sm - 1u) / blocks_per_sm));
+
+    unsigned serving = own, serving_len = own_len;
+    bool first = true, exhausted = false;
+    while (true) {
+        if (threadIdx.x < 32) {
+            unsigned n = 0u;
+            if (!exhausted) n = claim_from(sl, serving, serving_len, batch, first && serving == own, sh_tiles, exhausted);
+            first = false;
+            if (n == 0u) {
+                // This list is done.  If every non-empty list has a block on its SM, those blocks will
+                // finish them and this block may leave; otherwise adopt a list nobody is serving.
+                unsigned served = 0u;
+                if (own_len == 0u) __nanosleep(500);              // helpers: let the owners announce themselves first
+                if (threadIdx.x == 0) served = ld_volatile_u32(sl.ctl);
+                served = __shfl_sync(0xFFFFFFFFu, served, 0);
+                if (served < sl.nonempty) {
+                    const unsigned orphan = find_orphan(sl, own);
+                    if (orphan != 0xFFFFFFFFu) {
+                        serving = orphan;
+                        serving_len = sl.off[orphan + 1] - sl.off[orphan];
+                        n = claim_from(sl, serving, serving_len, batch, false, sh_tiles, exhausted);
+                        if (n == 0u) { n = 0xFFFFFFFFu; exhausted = true; }      // lost the race for it: look again
+                    }
+                }
+            }
+            if (threadIdx.x == 0) sh_n = n;
+        }
+        __syncthreads();
+        const unsigned n = sh_n;
+        if (n == 0u) break;
+        if (n != 0xFFFFFFFFu) {
+            for (unsigned i = 0; i < n; ++i) {
+                const size_t tile = sh_tiles[i];
+#pragma unroll
+                for (int sub = 0; sub < kSplit; ++sub) oneshot_group<N, C>(p, nvec, tile, sub * C);
+            }
+        }
+        __syncthreads();
+    }
+    pdl_trigger();
+    const size_t tail0 = nvec * kVecElems;
+    if (tail0 < count) {
+        for (int d = blockIdx.x; d < N; d += gridDim.x) {
+            const size_t e = tail0 + threadIdx.x;
+            if (e < count) reinterpret_cast<uint16_t*>(p.dst[d])[e] = fold_scalar<N>(p, e);
+        }
+    }
+    // the last block out rewinds cursors, presence flags and counters for the next launch
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(sl.ctl + 1, 1u) == gridDim.x - 1u) {
+            for (int s = 0; s < sl.num_sms; ++s) { sl.cursor[s] = 0u; sl.present[s] = 0u; }
+            sl.ctl[0] = 0u;
+            sl.ctl[1] = 0u;
+            __threadfence();
+        }
+    }
+}
+
 // ---- reduce-scatter: work item = (rank r, tile of shard r) -------------------------------------
 //
 // dst[r][j] = fold_k src[k][r*S + j].  `shard_vec` = S/8 (vector path requires S % 8 == 0, which

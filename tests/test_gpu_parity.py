@@ -58,7 +58,7 @@ COUNTS = [1, 7, 8, 9, 15, 16, 17, 2047, 2048, 2049, 4096, 6151, 100003, 262144]
 
 
 @pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16])
-@pytest.mark.parametrize("algo", ["oneshot", "oneshot_aware", "twoshot", "twoshot_put"])
+@pytest.mark.parametrize("algo", ["oneshot", "oneshot_aware", "oneshot_sm_lists", "twoshot", "twoshot_put"])
 def test_allreduce_special_values_all_counts(n, algo):
     for count in COUNTS:
         src = workloads.special_values(n, count, seed=1000 * n + count % 997)
@@ -68,6 +68,8 @@ def test_allreduce_special_values_all_counts(n, algo):
             nb.nuna_allreduce_oneshot(dsrc, dst.view, count)
         elif algo == "oneshot_aware":
             nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE)
+        elif algo == "oneshot_sm_lists":
+            nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS)
         else:
             nb.nuna_allreduce_twoshot(dsrc, dst.view, count, flags=nb.NUNA_TWOSHOT_PUT if algo == "twoshot_put" else 0)
         got = dst.numpy()
@@ -256,6 +258,42 @@ def test_chain_nodes_are_ordered_even_with_dependent_launch(flags):
                     assert float(v.min()) == expect and float(v.max()) == expect
     finally:
         nb.nuna_chain_destroy(chain)
+
+
+def test_sm_lists_replay_and_after_probe():
+    """The work-list kernel rewinds its own cursors: graph replays and repeated calls stay correct, with
+    the one-domain plan (no probe yet in this process is not guaranteed, so both orders are exercised)."""
+    flags = nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS
+    for n, count in ((8, 32 * 8192), (8, 4096), (3, 100003), (16, 1 << 20)):
+        src = workloads.special_values(n, count, seed=n + count % 89)
+        want = oracle.allreduce(src, nthreads=4)[0]
+        dsrc = upload(src)
+        dst = [torch.zeros(count, dtype=torch.int16, device="cuda") for _ in range(n)]
+        nb.nuna_allreduce_oneshot(dsrc, dst, count, flags=flags)              # builds the plan (allocates)
+        g = torch.cuda.CUDAGraph()
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            with torch.cuda.graph(g, stream=s):
+                nb.nuna_allreduce_oneshot(dsrc, dst, count, flags=flags, stream=s)
+                nb.nuna_allreduce_oneshot(dsrc, dst, count, flags=flags | nb.NUNA_LAUNCH_PDL, stream=s)
+        for _ in range(4):
+            for t in dst:
+                t.fill_(-1)
+            g.replay()
+            torch.cuda.synchronize()
+            for t in dst:
+                assert_same_bits(t.cpu().numpy().view(np.uint16), want, f"sm lists n={n} count={count}")
+    # after a probe the plan uses two domains: new shapes get new plans, results stay the same
+    probe_bufs = [torch.zeros(1 << 16, dtype=torch.int16, device="cuda") for _ in range(4)]
+    nb.nuna_probe_topology(probe_bufs)
+    for n, count in ((8, 64 * 8192), (8, 2048 + 8), (5, 33333)):
+        src = workloads.special_values(n, count, seed=count)
+        want = oracle.allreduce(src, nthreads=4)[0]
+        dst = Dst(n, count)
+        for _ in range(3):
+            nb.nuna_allreduce_oneshot(upload(src), dst.view, count, flags=flags)
+        for got in dst.numpy():
+            assert_same_bits(got, want, "sm lists after probe")
 
 
 def test_host_buffer_entry_point():
