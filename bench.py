@@ -134,18 +134,12 @@ class ClockSampler:
 def run_gpu(args):
     import numpy as np
     import torch
-    import torch.distributed as dist
-
     from paper_2608_00867_b200 import binding as nb
     from paper_2608_00867_b200 import workloads
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    from paper_2608_00867_b200.replicas import Replicas
+    rep = Replicas(backend="nccl")
+    rank, world, local = rep.rank, rep.world, rep.local
 
     peak_gbs, peak_src = measured_peaks()
     l2 = torch.cuda.get_device_properties(local).L2_cache_size
@@ -156,17 +150,7 @@ def run_gpu(args):
     if rank == 0:
         sampler.start()
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    barrier, max_over_ranks = rep.barrier, rep.max_over_ranks
 
     def make_sets(n, count, dst_count, min_bytes, dist_name="normal", seed=1, max_sets=4096):
         """Device buffer sets whose total footprint exceeds min_bytes (cold protocol).
@@ -379,8 +363,7 @@ def run_gpu(args):
     launches_total = nb.nuna_launch_count()
     status = nb.nuna_device_status()
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        dist.destroy_process_group()
+    rep.close()
     if rank != 0:
         return 0
 

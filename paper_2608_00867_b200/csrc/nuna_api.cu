@@ -136,9 +136,15 @@ static int occupancy(Context* c, K kernel, int* cache)
     return *cache;
 }
 
-static unsigned pick_grid(const Context* c, size_t nitems, int blocks_per_sm)
+// Grid size: `waves` x (SMs x resident blocks per SM), never more than the work items.  Streaming
+// kernels (two-shot put, reduce-scatter, allgather) run one item per block (waves = 0: no cap): leaving
+// the balancing to the hardware block scheduler measured 0.99 of the copy peak at 64 MiB per rank
+// against 0.90 for a persistent grid-stride loop.  The one-shot wants its N readers of a tile close in
+// time so that re-reads hit L2: four waves measured best (0.70 of peak at 64 MiB against 0.63 for one
+// wave and 0.62 for an uncapped grid).
+static unsigned pick_grid(const Context* c, size_t nitems, int blocks_per_sm, int waves = 1)
 {
-    size_t cap = (size_t)c->num_sms * (size_t)blocks_per_sm;
+    size_t cap = waves > 0 ? (size_t)c->num_sms * (size_t)blocks_per_sm * (size_t)waves : ((size_t)1 << 22);
     if (c->blocks_override > 0) cap = (size_t)c->blocks_override;
     return (unsigned)std::max<size_t>(1, std::min(nitems, cap));
 }
@@ -424,7 +430,8 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsi
         auto k = k_oneshot_rr<N, U>;
         const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
         const size_t nitems = std::max<size_t>(ntiles * N, (count % kVecElems) ? (size_t)N : 0);
-        const unsigned grid = pick_grid(c, nitems, occupancy(c, k, &occ));
+        // one resident wave while the message is small enough for latency to matter, four beyond
+        const unsigned grid = pick_grid(c, nitems, occupancy(c, k, &occ), count * 2 >= ((size_t)8 << 20) ? 4 : 1);
         return launch(k, grid, stream, mode, p, count, ntiles);
     });
 }
@@ -439,7 +446,7 @@ int launch_twoshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsi
             static int occ = 0;
             auto k = k_twoshot_put<N, U>;
             const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
-            const unsigned grid = pick_grid(c, std::max<size_t>(ntiles, 1), occupancy(c, k, &occ));
+            const unsigned grid = pick_grid(c, std::max<size_t>(ntiles, 1), occupancy(c, k, &occ), 0);
             return launch(k, grid, stream, mode, p, count, ntiles);
         });
     }
@@ -475,7 +482,7 @@ int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shar
         static int occ = 0;
         auto k = k_reduce_scatter<N, U>;
         const size_t tiles = ceil_div(shard_vec, (size_t)kThreads * U);
-        const unsigned grid = pick_grid(c, tiles * N, occupancy(c, k, &occ));
+        const unsigned grid = pick_grid(c, tiles * N, occupancy(c, k, &occ), 0);
         return launch(k, grid, stream, mode, p, shard_vec, tiles);
     });
 }
@@ -492,7 +499,7 @@ int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, un
     constexpr int U = 2;
     auto k = k_allgather<U>;
     const size_t tiles = ceil_div(shard_vec, (size_t)kThreads * U);
-    const unsigned grid = pick_grid(c, tiles * nranks, occupancy(c, k, &occ));
+    const unsigned grid = pick_grid(c, tiles * nranks, occupancy(c, k, &occ), 0);
     return launch(k, grid, stream, mode, p, nranks, shard_vec, tiles);
 }
 
