@@ -524,6 +524,8 @@ __device__ __forceinline__ bool flag_barrier(BarrierWords* bw, unsigned int expe
         asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(&bw->arrive) : "memory");
         if (prev == expected - 1) {
             bw->arrive = 0;                            // nobody touches it again before the epoch moves
+            bw->work[0] = 0;                           // everyone is past phase 1 and nobody is in phase 2 yet:
+            bw->work[1] = 0;                           // rewind both work cursors for this phase 2 / the next launch
             asm volatile("red.release.gpu.global.add.u32 [%0], 1;" :: "l"(&bw->epoch) : "memory");
         } else {
             const unsigned long long t0 = globaltimer_ns();
@@ -557,17 +559,35 @@ k_twoshot_fused(const RankPtrs p, uint4* scratch, const size_t count, const size
     const size_t nvec = count / kVecElems;
     const size_t tiles_per_chunk = (chunk_vec + kThreads * U - 1) / (kThreads * U);
     const size_t nitems = tiles_per_chunk * N;
+    __shared__ unsigned sh_item;
     unsigned int epoch0 = 0;
     if (threadIdx.x == 0) epoch0 = ld_acquire(&bw->epoch);
 
-    for (size_t item = blockIdx.x; item < nitems; item += gridDim.x) {
+    // Work distribution inside the persistent grid: a block's first item is its own index (no latency
+    // at start), every further item is claimed from a device-wide cursor, the next claim being issued
+    // before the current item is processed.  Static striding left the blocks of the die with more SMs
+    // behind (its SMs share the same memory bandwidth among more blocks); claiming evens that out.
+    auto for_each_item = [&](unsigned int* cursor, auto&& body) {
+        size_t item = blockIdx.x;
+        unsigned next = 0;
+        while (item < nitems) {
+            if (threadIdx.x == 0) next = atomicAdd(cursor, 1u);
+            body(item);
+            if (threadIdx.x == 0) sh_item = next;
+            __syncthreads();
+            item = (size_t)gridDim.x + sh_item;
+            __syncthreads();
+        }
+    };
+
+    for_each_item(&bw->work[0], [&](size_t item) {
         const int r = (int)(item % N);                 // rank fastest: neighbouring blocks work on different chunks
         const size_t tile = item / N;
         const size_t off = (size_t)r * chunk_vec;
-        if (off >= nvec) continue;
+        if (off >= nvec) return;
         const size_t len = (nvec - off < chunk_vec) ? nvec - off : chunk_vec;
         reduce_tile<N, U>(p, scratch + off, off, len, tile);
-    }
+    });
     const size_t tail0 = nvec * kVecElems;             // ragged tail: reduced by block 0 into scratch
     if (tail0 < count && blockIdx.x == 0) {
         const size_t e = tail0 + threadIdx.x;
@@ -576,14 +596,14 @@ k_twoshot_fused(const RankPtrs p, uint4* scratch, const size_t count, const size
 
     if (!flag_barrier(bw, gridDim.x, epoch0, timeout_ns)) return;
 
-    for (size_t item = blockIdx.x; item < nitems; item += gridDim.x) {
+    for_each_item(&bw->work[1], [&](size_t item) {
         const int r = (int)(item % N);
         const size_t tile = item / N;
         const size_t off = (size_t)r * chunk_vec;
-        if (off >= nvec) continue;
+        if (off >= nvec) return;
         const size_t len = (nvec - off < chunk_vec) ? nvec - off : chunk_vec;
         gather_tile<U>(scratch + off, p, N, off, len, tile, true);
-    }
+    });
     if (tail0 < count && blockIdx.x == 0) {
         const size_t e = tail0 + threadIdx.x;
         if (e < count) {

@@ -20,7 +20,8 @@ struct BarrierWords {
     unsigned int arrive;
     unsigned int epoch;
     unsigned int status;
-    unsigned int pad;
+    unsigned int work[2];     // dynamic work cursors of the fused two-shot's two phases (zero between launches)
+    unsigned int pad[3];
 };
 
 }  // namespace nuna
