@@ -43,7 +43,7 @@ def _load():
         lib = ctypes.CDLL(build())
         pp = ctypes.POINTER(ctypes.c_void_p)
         for name in ("nuna_oracle_allreduce_bf16", "nuna_oracle_reduce_scatter_bf16",
-                     "nuna_oracle_allgather_bf16"):
+                     "nuna_oracle_allgather_bf16", "nuna_oracle_alltoall_bf16"):
             fn = getattr(lib, name)
             fn.argtypes = [pp, pp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int]
             fn.restype = None
@@ -103,6 +103,18 @@ def allgather(src: Sequence[np.ndarray], nthreads: int = 1) -> List[np.ndarray]:
     src = [np.ascontiguousarray(a) for a in src]
     dst = [np.empty(n * shard, dtype=np.uint16) for _ in range(n)]
     _load().nuna_oracle_allgather_bf16(_ptrs(src), _ptrs(dst), n, shard, int(nthreads))
+    return dst
+
+
+def alltoall(src: Sequence[np.ndarray], nthreads: int = 1) -> List[np.ndarray]:
+    """``src[r]`` holds N blocks of S elements (block d goes to rank d); returns N arrays of ``N*S``."""
+    n, total = len(src), len(src[0])
+    _check_src(src, total)
+    if total % n:
+        raise ValueError("source length must be a multiple of the rank count")
+    src = [np.ascontiguousarray(a) for a in src]
+    dst = [np.empty(total, dtype=np.uint16) for _ in range(n)]
+    _load().nuna_oracle_alltoall_bf16(_ptrs(src), _ptrs(dst), n, total // n, int(nthreads))
     return dst
 
 

@@ -20,6 +20,7 @@
  *   allreduce      dst[d][i]       = rne((((f(src[0][i]) + f(src[1][i])) + ...) + f(src[N-1][i])))
  *   reduce_scatter dst[r][j]       = the same fold over src[0..N-1][r*S + j]
  *   allgather      dst[d][r*S + j] = src[r][j]                          (16-bit copy)
+ *   alltoall       dst[d][r*S + j] = src[r][d*S + j]                    (16-bit copy)
  *
  * The accumulator starts from f(src[0][i]), not from +0, so N values take N-1
  * additions and an all-(-0) column stays -0.  Every partial sum is a binary32
@@ -107,6 +108,22 @@ void nuna_oracle_allgather_bf16(const uint16_t *const *src, uint16_t *const *dst
 #pragma omp parallel for schedule(static) num_threads(nthreads) if (nthreads > 1)
             for (size_t j = 0; j < shard; ++j)
                 dst[d][(size_t)r * shard + j] = src[r][j];
+        }
+}
+
+/* alltoall (Section 2.1: token routing between experts, the paper's third collective): src[r] holds
+ * nranks blocks of `block` elements, block d being what rank r sends to rank d; dst[d] holds nranks
+ * blocks, block r being what it received from rank r.  dst[d][r*block + i] = src[r][d*block + i],
+ * a 16-bit copy. */
+void nuna_oracle_alltoall_bf16(const uint16_t *const *src, uint16_t *const *dst,
+                               int nranks, size_t block, int nthreads)
+{
+    (void)nthreads;
+    for (int d = 0; d < nranks; ++d)
+        for (int r = 0; r < nranks; ++r) {
+#pragma omp parallel for schedule(static) num_threads(nthreads) if (nthreads > 1)
+            for (size_t i = 0; i < block; ++i)
+                dst[d][(size_t)r * block + i] = src[r][(size_t)d * block + i];
         }
 }
 

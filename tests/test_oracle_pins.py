@@ -254,3 +254,31 @@ def test_empty_and_single():
     one = u16(0x3F80, 0xFFFF, 0x8000)
     assert np.array_equal(oracle.allreduce([one])[0][[0, 2]], one[[0, 2]])
     assert np.array_equal(oracle.allgather([one])[0], one)
+
+
+# ---- alltoall: a block transpose of raw bits -----------------------------------------------------------
+
+def test_alltoall_is_the_block_transpose():
+    n, block = 5, 37
+    rng = np.random.Generator(np.random.PCG64(6))
+    src = [rng.integers(0, 1 << 16, size=n * block, dtype=np.uint32).astype(np.uint16) for _ in range(n)]
+    out = oracle.alltoall(src)
+    cube = np.stack([s.reshape(n, block) for s in src])          # [sender r][receiver d][i]
+    want = cube.transpose(1, 0, 2)                               # [receiver d][sender r][i]  (numpy's own transpose)
+    for d in range(n):
+        assert np.array_equal(out[d], want[d].reshape(-1))
+    # applying it twice returns every buffer to where it started
+    back = oracle.alltoall(out)
+    for r in range(n):
+        assert np.array_equal(back[r], src[r])
+
+
+def test_alltoall_of_replicated_blocks_is_allgather():
+    n, block = 4, 64
+    shards = workloads.rank_buffers(n, block, "uniform", seed=2)
+    src = [np.tile(s, n) for s in shards]                        # rank r sends the same block to everyone
+    a2a, ag = oracle.alltoall(src), oracle.allgather(shards)
+    for d in range(n):
+        assert np.array_equal(a2a[d], ag[d])
+    assert np.array_equal(oracle.alltoall([shards[0]])[0], shards[0])   # one rank: identity
+    assert np.array_equal(oracle.alltoall(src, 1)[2], oracle.alltoall(src, 8)[2])
