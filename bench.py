@@ -274,7 +274,7 @@ def run_gpu(args):
         extras["e2e"] = {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": N_RANKS * w.bytes_per_rank,
                          "d2h_bytes_per_step": N_RANKS * w.bytes_per_rank}
 
-    sweep, ag_row, chain_rows = [], None, []
+    sweep, ag_row, a2a_row, chain_rows = [], None, None, []
     if not args.quick:
         # ---- message-size sweep, 8 ranks, 8 KiB .. 64 MiB per rank --------------------------------------
         algos = {
@@ -310,6 +310,17 @@ def run_gpu(args):
         ag_row = {"workload": wa.name, "us": round(ag_us, 3), "algorithmic_bytes": ag_bytes,
                   "gbs": round(ag_bytes / ag_us / 1e3, 1), "frac_of_peak": round(ag_bytes / ag_us / 1e3 / peak_gbs, 4)}
         del asets
+        torch.cuda.empty_cache()
+
+        # ---- alltoall, 8 ranks x 64 KiB per pair ----------------------------------------------------------
+        wt = workloads.config_alltoall8()
+        tsets = make_sets(wt.nranks, wt.count, wt.count, 2 * l2 + (64 << 20), "normal", wt.seed)
+        blk = wt.count // wt.nranks
+        a2a_us = per_call_us(lambda s, d, st: nb.nuna_alltoall(s, d, blk, stream=st), tsets, 512, 3)
+        a2a_bytes = 2 * wt.nranks * wt.bytes_per_rank
+        a2a_row = {"workload": wt.name, "us": round(a2a_us, 3), "algorithmic_bytes": a2a_bytes,
+                   "gbs": round(a2a_bytes / a2a_us / 1e3, 1), "frac_of_peak": round(a2a_bytes / a2a_us / 1e3 / peak_gbs, 4)}
+        del tsets
         torch.cuda.empty_cache()
 
         # ---- decode-step chain: 160 back-to-back one-shot allreduces in one graph ------------------------
@@ -389,7 +400,7 @@ def run_gpu(args):
         "launches_since_load": int(launches_total),
         "device_status": status,
         "clocks": clocks,
-        "sweep": sweep, "allgather16": ag_row, "decode_chain": chain_rows,
+        "sweep": sweep, "allgather16": ag_row, "alltoall8": a2a_row, "decode_chain": chain_rows,
     }
     line.update(extras)
     if cpu is not None:

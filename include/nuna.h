@@ -198,6 +198,13 @@ int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks,
 int nuna_allgather(const void* const* src, void* const* dst, int nranks,
                    size_t shard_count, int dtype, unsigned flags, void* stream);
 
+/* Alltoall (Section 2.1: expert token routing, the paper's third collective): src[r] holds nranks blocks
+ * of block_count elements, block d being what rank r sends to rank d; dst[d] holds nranks blocks, block
+ * r being what it received from rank r: dst[d][r*block_count + i] = src[r][d*block_count + i], copied
+ * bit for bit.  Placement bits of `flags` are accepted and ignored (every block is touched once).      */
+int nuna_alltoall(const void* const* src, void* const* dst, int nranks,
+                  size_t block_count, int dtype, unsigned flags, void* stream);
+
 /* Two-shot allreduce for callers that must not allocate device memory.  (The paper has no counterpart:
  * this is a deployment convenience of the library.)  Some hosts of this code cannot call cudaMalloc
  * on the request path: an inference server that has handed the whole GPU to its own memory pool, where

@@ -86,7 +86,8 @@ def lib() -> ctypes.CDLL:
         L = ctypes.CDLL(_LIB_PATH)
         vpp = ctypes.POINTER(ctypes.c_void_p)
         coll = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint, ctypes.c_void_p]
-        for name in ("nuna_allreduce_oneshot", "nuna_allreduce_twoshot", "nuna_reduce_scatter", "nuna_allgather"):
+        for name in ("nuna_allreduce_oneshot", "nuna_allreduce_twoshot", "nuna_reduce_scatter", "nuna_allgather",
+                     "nuna_alltoall"):
             getattr(L, name).argtypes = coll
             getattr(L, name).restype = ctypes.c_int
         L.nuna_allreduce_twoshot_static.argtypes = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_void_p]
@@ -184,6 +185,10 @@ def nuna_reduce_scatter(src, dst, shard_count, dtype=NUNA_BF16, flags=0, stream=
 
 def nuna_allgather(src, dst, shard_count, dtype=NUNA_BF16, flags=0, stream=None, check=True, nranks=None) -> int:
     return _collective("nuna_allgather", src, dst, shard_count, dtype, flags, stream, check, nranks)
+
+
+def nuna_alltoall(src, dst, block_count, dtype=NUNA_BF16, flags=0, stream=None, check=True, nranks=None) -> int:
+    return _collective("nuna_alltoall", src, dst, block_count, dtype, flags, stream, check, nranks)
 
 
 NUNA_STATIC_MAX_COUNT = 2 * 1024 * 1024

@@ -440,9 +440,14 @@ k_reduce_scatter_scalar(const RankPtrs p, const size_t shard)
     }
 }
 
-// ---- allgather: work item = (rank r, tile of shard r); local load, store to all N -----------------
+// ---- allgather: work item = (rank r, tile of shard r, group of destinations); local load, remote store ----
+//
+// The paper's form (Figure "Allocation_Diagram"): a thread block loads a chunk of its own rank's
+// buffer and stores it into the peers' buffers.  `dsplit` blocks share one tile, each storing to
+// nranks / dsplit destinations: small messages need the extra blocks to fill the machine (N stores per
+// load from one thread are issue-bound), large ones use dsplit = 1 and read every source byte once.
 template <int U>
-__device__ __forceinline__ void gather_tile(const uint4* in, const RankPtrs& p, int nranks, size_t dst_off_vec,
+__device__ __forceinline__ void gather_tile(const uint4* in, const RankPtrs& p, int d0, int d1, size_t dst_off_vec,
                                             size_t nvec, size_t tile, bool coherent)
 {
     const size_t base = tile * (size_t)(kThreads * U) + threadIdx.x;
@@ -456,21 +461,25 @@ __device__ __forceinline__ void gather_tile(const uint4* in, const RankPtrs& p, 
     for (int u = 0; u < U; ++u) {
         const size_t i = base + (size_t)u * kThreads;
         if (i < nvec) {
-            for (int d = 0; d < nranks; ++d) st_dst(p.dst[d] + dst_off_vec + i, v[u]);
+            for (int d = d0; d < d1; ++d) st_dst(p.dst[d] + dst_off_vec + i, v[u]);
         }
     }
 }
 
 template <int U>
 __global__ void __launch_bounds__(kThreads, min_blocks(U))
-k_allgather(const RankPtrs p, const int nranks, const size_t shard_vec, const size_t tiles_per_shard)
+k_allgather(const RankPtrs p, const int nranks, const size_t shard_vec, const size_t tiles_per_shard, const int dsplit)
 {
     pdl_wait();
-    const size_t nitems = tiles_per_shard * nranks;
+    const int per = (nranks + dsplit - 1) / dsplit;
+    const size_t nitems = tiles_per_shard * nranks * dsplit;
     for (size_t item = blockIdx.x; item < nitems; item += gridDim.x) {
-        const int r = (int)(item / tiles_per_shard);
-        const size_t tile = item % tiles_per_shard;
-        gather_tile<U>(p.src[r], p, nranks, (size_t)r * shard_vec, shard_vec, tile, false);
+        const int g = (int)(item % dsplit);
+        const size_t rt = item / dsplit;
+        const int r = (int)(rt % nranks);
+        const size_t tile = rt / nranks;
+        const int d0 = g * per, d1 = min(nranks, d0 + per);
+        gather_tile<U>(p.src[r], p, d0, d1, (size_t)r * shard_vec, shard_vec, tile, false);
     }
     pdl_trigger();
 }
@@ -485,6 +494,54 @@ k_allgather_scalar(const RankPtrs p, const int nranks, const size_t shard)
         const uint16_t v = ld_src16(reinterpret_cast<const uint16_t*>(p.src[r]) + (e - (size_t)r * shard));
         for (int d = 0; d < nranks; ++d) reinterpret_cast<uint16_t*>(p.dst[d])[e] = v;
     }
+}
+
+// ---- alltoall: work item = (sender r, receiver d, tile of the block r sends to d) -------------------------
+//
+// dst[d][r*S + j] = src[r][d*S + j]: the paper's third collective (expert token routing), a block
+// transpose.  Local load from the sender's buffer, store into the receiver's (the put form).
+template <int U>
+__global__ void __launch_bounds__(kThreads, min_blocks(U))
+k_alltoall(const RankPtrs p, const int nranks, const size_t block_vec, const size_t tiles_per_block)
+{
+    pdl_wait();
+    const size_t pairs = (size_t)nranks * nranks;
+    const size_t nitems = tiles_per_block * pairs;
+    for (size_t item = blockIdx.x; item < nitems; item += gridDim.x) {
+        const size_t pair = item % pairs, tile = item / pairs;   // pairs fastest: neighbours hit different buffers
+        const int r = (int)(pair / nranks), d = (int)(pair % nranks);
+        const uint4* in = p.src[r] + (size_t)d * block_vec;
+        uint4* out = p.dst[d] + (size_t)r * block_vec;
+        const size_t base = tile * (size_t)(kThreads * U) + threadIdx.x;
+        uint4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t i = base + (size_t)u * kThreads;
+            if (i < block_vec) v[u] = ld_src(in + i);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t i = base + (size_t)u * kThreads;
+            if (i < block_vec) st_dst(out + i, v[u]);
+        }
+    }
+    pdl_trigger();
+}
+
+// Any block length (used when S % 8 != 0): one element per thread.
+__global__ void __launch_bounds__(kThreads)
+k_alltoall_scalar(const RankPtrs p, const int nranks, const size_t block)
+{
+    pdl_wait();
+    const size_t per_rank = block * nranks, total = per_rank * nranks;
+    for (size_t e = (size_t)blockIdx.x * kThreads + threadIdx.x; e < total; e += (size_t)gridDim.x * kThreads) {
+        const int d = (int)(e / per_rank);
+        const size_t within = e - (size_t)d * per_rank;
+        const int r = (int)(within / block);
+        const size_t i = within - (size_t)r * block;
+        reinterpret_cast<uint16_t*>(p.dst[d])[within] = ld_src16(reinterpret_cast<const uint16_t*>(p.src[r]) + (size_t)d * block + i);
+    }
+    pdl_trigger();
 }
 
 // ---- flag barrier among the co-resident blocks of one launch ----------------------------------------
@@ -602,7 +659,7 @@ k_twoshot_fused(const RankPtrs p, uint4* scratch, const size_t count, const size
         const size_t off = (size_t)r * chunk_vec;
         if (off >= nvec) return;
         const size_t len = (nvec - off < chunk_vec) ? nvec - off : chunk_vec;
-        gather_tile<U>(scratch + off, p, N, off, len, tile, true);
+        gather_tile<U>(scratch + off, p, 0, N, off, len, tile, true);
     });
     if (tail0 < count && blockIdx.x == 0) {
         const size_t e = tail0 + threadIdx.x;

@@ -86,6 +86,11 @@ def config_allgather16() -> Workload:
     return Workload("ag_n16_64KiB", "allgather", 16, 32768, "uniform", 3)
 
 
+def config_alltoall8() -> Workload:
+    """Expert token routing: eight ranks, 64 KiB per (sender, receiver) pair, 512 KiB per rank, N(0,1)."""
+    return Workload("a2a_n8_64KiB", "alltoall", 8, 8 * 32768, "normal", 6)
+
+
 def config_decode_chain(tokens: int) -> Workload:
     """One node of the decode-step chain: eight ranks, tokens x 8192 bf16, N(0,1)."""
     k = {1: 0, 8: 1, 64: 2, 256: 3}.get(tokens, 4)

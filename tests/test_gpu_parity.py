@@ -141,6 +141,23 @@ def test_config_allgather16_raw_bits():
             assert np.array_equal(got[d], want[d])
 
 
+@pytest.mark.parametrize("n,block", [(8, 4096), (8, 1000), (16, 33), (3, 8), (5, 2049), (8, 65536), (2, 1), (1, 77), (16, 8192)])
+def test_alltoall_raw_bits(n, block):
+    rng = np.random.Generator(np.random.PCG64(n * 1000 + block))
+    src = [rng.integers(0, 1 << 16, size=n * block, dtype=np.uint32).astype(np.uint16) for _ in range(n)]
+    want = oracle.alltoall(src, nthreads=4)
+    dst = Dst(n, n * block)
+    nb.nuna_alltoall(upload(src), dst.view, block)
+    got = dst.numpy()
+    for d in range(n):
+        assert np.array_equal(got[d], want[d]), (n, block, d)
+    # twice = identity
+    back = Dst(n, n * block)
+    nb.nuna_alltoall(dst.view, back.view, block, flags=nb.NUNA_LAUNCH_PDL)
+    for r, g in enumerate(back.numpy()):
+        assert np.array_equal(g, src[r])
+
+
 def test_sweep_sizes_one_and_two_shot_agree_with_oracle():
     for w in workloads.config_size_sweep(13, 22):
         src = workloads.make(w)
