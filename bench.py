@@ -214,7 +214,8 @@ def run_gpu(args):
     w = workloads.config_decode_activation()
     count = w.count
     sets = make_sets(N_RANKS, count, count, 2 * l2 + (64 << 20), "normal", w.seed)
-    oneshot = lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, count, flags=nb.NUNA_PLACE_AUTO, stream=st)
+    headline_flags = nb.NUNA_PLACE_AUTO | nb.NUNA_LAUNCH_PDL
+    oneshot = lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, count, flags=headline_flags, stream=st)
     K, W = args.steps, max(args.warmup, 3)
     nodes = min(K, 1000)
     replays, rem = divmod(K, nodes)
@@ -259,6 +260,46 @@ def run_gpu(args):
         place[pname] = {"cold_us": round(per_call_us(fn, sets, 1000, 3), 3),
                         "l2_resident_us": round(per_call_us(fn, sets[:1], 1000, 3), 3)}
     extras["placement_512KiB"] = place
+
+    # ---- robustness to concurrent work (the paper runs its collectives beside a GEMM, Section 6.6) ------------
+    # 1 MiB per rank one-shot, L2-resident sources, while a second stream runs (a) nothing, (b) a streaming
+    # copy, (c) a dense bf16 matmul (a library GEMM used only as a load generator).
+    if not args.quick:
+        c1 = (1 << 20) // 2
+        isets = make_sets(N_RANKS, c1, c1, 0, "normal", 77, max_sets=2)
+        side = torch.cuda.Stream()
+        big_a = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        big_b = torch.empty_like(big_a)
+        ma = torch.randn(4096, 4096, device="cuda", dtype=torch.bfloat16)
+        mb = torch.randn(4096, 4096, device="cuda", dtype=torch.bfloat16)
+        loads = {"idle": None, "streaming_copy": lambda: big_b.copy_(big_a), "bf16_gemm_4096": lambda: torch.matmul(ma, mb)}
+        inter = {}
+        for lname, load in loads.items():
+            row = {}
+            for pname, pflags in (("roundrobin", nb.NUNA_PLACE_ROUNDROBIN), ("aware_colocated", nb.NUNA_PLACE_AWARE)):
+                fn = lambda s, d, st, f=pflags: nb.nuna_allreduce_oneshot(s, d, c1, flags=f, stream=st)
+                g = capture(fn, isets, 400)
+                with torch.cuda.stream(stream):
+                    g.replay()
+                torch.cuda.synchronize()
+                if load is not None:                       # enqueue the background work, then time beside it
+                    with torch.cuda.stream(side):
+                        for _ in range(80):
+                            load()
+                with torch.cuda.stream(stream):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    g.replay()
+                    g.replay()
+                    e1.record(stream)
+                busy = (not side.query()) if load is not None else None   # background still running at the end?
+                torch.cuda.synchronize()
+                row[pname] = {"us": round(e0.elapsed_time(e1) * 1e3 / 800, 3), "background_outlasted_timing": busy}
+                del g
+            inter[lname] = row
+        extras["interference_1MiB_resident"] = inter
+        del isets, big_a, big_b, ma, mb
+        torch.cuda.empty_cache()
     if True:
         # ---- end to end through the host-buffer entry point (pinned host memory) -----------------------
         hsrc = [torch.from_numpy(a.view(np.int16).copy()).pin_memory() for a in workloads.make(w)]
@@ -388,7 +429,8 @@ def run_gpu(args):
         "ms_per_step": us_per_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 storage, f32 accumulate", "data": "synthetic",
         "config": {"workload": w.name, "nranks": N_RANKS, "bytes_per_rank": w.bytes_per_rank,
-                   "algorithm": "one-shot allreduce, placement AUTO", "launch": "CUDA graph of back-to-back calls",
+                   "algorithm": "one-shot allreduce, placement AUTO, programmatic dependent launch",
+                   "launch": "CUDA graph of back-to-back calls",
                    "l2_protocol": f"cold: rotates over {len(sets)} buffer sets ({len(sets) * 2 * N_RANKS * w.bytes_per_rank >> 20} MiB) > 2 x L2",
                    "multi_gpu": "independent replicas (the emulated collective has no inter-GPU step)"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,

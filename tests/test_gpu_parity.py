@@ -253,6 +253,28 @@ def test_chain_every_node_matches_oracle(flags, two_shot):
     assert nb.nuna_device_status() == nb.NUNA_OK
 
 
+@pytest.mark.parametrize("tokens", [1, 8, 256])
+def test_decode_chain_160_nodes_as_benchmarked(tokens):
+    """The benchmark's chain: 160 nodes over two alternating buffer sets, AUTO placement under the
+    resident hint, dependent launch.  Every node's destinations are checked (each set is written 80 times)."""
+    w = workloads.config_decode_chain(tokens)
+    flags = nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT | nb.NUNA_LAUNCH_PDL
+    srcs = [workloads.rank_buffers(w.nranks, w.count, "normal", seed=w.seed + s) for s in range(2)]
+    want = [oracle.allreduce(s, nthreads=8)[0] for s in srcs]
+    dsrc = [upload(s) for s in srcs]
+    ddst = [[torch.zeros(w.count, dtype=torch.int16, device="cuda") for _ in range(w.nranks)] for _ in range(2)]
+    chain = nb.nuna_chain_create(dsrc, ddst, workloads.CHAIN_NODES, w.count, flags=flags)
+    try:
+        for _ in range(2):
+            nb.nuna_chain_launch(chain)
+        torch.cuda.synchronize()
+        for s in range(2):
+            for t in ddst[s]:
+                assert np.array_equal(t.cpu().numpy().view(np.uint16), want[s])
+    finally:
+        nb.nuna_chain_destroy(chain)
+
+
 @pytest.mark.parametrize("flags", [0, nb.NUNA_LAUNCH_PDL, nb.NUNA_LAUNCH_PDL | nb.NUNA_PLACE_AWARE])
 def test_chain_nodes_are_ordered_even_with_dependent_launch(flags):
     """Node k+1 reads what node k wrote: ones -> 8 -> 64 -> 512 -> 4096 only if every node waited."""
