@@ -252,7 +252,18 @@ def run_gpu(args):
     extras = {}
     # ---- placement on the headline workload: round-robin baseline vs the two placement-aware kernels ---------
     # (per-SM work lists use the topology of a probe run here on the first buffer set)
-    nb.nuna_probe_topology(list(sets[0][0]) + list(sets[0][1]))
+    topo = nb.nuna_probe_topology(list(sets[0][0]) + list(sets[0][1]))
+    doms = [topo.sm_domain[s] for s in range(topo.num_sms)]
+    extras["probe"] = {
+        "sms": topo.num_sms, "sms_reported": topo.sms_reported, "lines": topo.num_lines,
+        "verdict": "nonuniform" if topo.verdict == nb.NUNA_TOPO_NONUNIFORM else "uniform",
+        "domain_sizes": [doms.count(0), doms.count(1)], "near_cycles": round(topo.near_lat, 1),
+        "far_cycles": round(topo.far_lat, 1), "gap_cycles": round(topo.domain_gap, 1), "noise_cycles": round(topo.noise, 2),
+        "sm_mean_hit_cycles_min_max": [round(min(topo.sm_lat_hit[:topo.num_sms]), 1), round(max(topo.sm_lat_hit[:topo.num_sms]), 1)],
+        "sm_miss_cycles_min_max": [round(min(topo.sm_lat_miss[:topo.num_sms]), 1), round(max(topo.sm_lat_miss[:topo.num_sms]), 1)],
+        "hist_first_cycle": nb.NUNA_HIST_FIRST, "hist_step": nb.NUNA_HIST_STEP,
+        "hist_near": list(topo.hist_near), "hist_far": list(topo.hist_far),
+    }
     place = {}
     for pname, pflags in (("roundrobin", nb.NUNA_PLACE_ROUNDROBIN), ("aware_colocated", nb.NUNA_PLACE_AWARE),
                           ("aware_sm_lists", nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS)):
@@ -298,6 +309,18 @@ def run_gpu(args):
                 del g
             inter[lname] = row
         extras["interference_1MiB_resident"] = inter
+
+        # ---- sensitivity to the number of thread blocks (the paper contrasts few and many, Section 6.5) ---------
+        blocks_rows = {}
+        for label, fn_of in (("oneshot_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c1, stream=st))),
+                             ("twoshot_put_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c1, flags=nb.NUNA_TWOSHOT_PUT, stream=st)))):
+            row = {}
+            for blocks in (8, 37, 148, 592, 0):
+                nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, blocks)
+                row["default" if blocks == 0 else str(blocks)] = round(per_call_us(fn_of(), isets, 200, 2), 3)
+            nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, 0)
+            blocks_rows[label] = row
+        extras["blocks_sensitivity_resident_us"] = blocks_rows
         del isets, big_a, big_b, ma, mb
         torch.cuda.empty_cache()
     if True:

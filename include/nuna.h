@@ -96,6 +96,9 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* on
 #define NUNA_MAX_PROBE_LINES  2048
 #define NUNA_TOPO_UNIFORM     0
 #define NUNA_TOPO_NONUNIFORM  1
+#define NUNA_HIST_BINS        48
+#define NUNA_HIST_FIRST       200
+#define NUNA_HIST_STEP        4
 
 typedef struct nuna_topology {
     int num_sms;                     /* cudaDeviceProp.multiProcessorCount                                 */
@@ -121,6 +124,13 @@ typedef struct nuna_topology {
     unsigned char line_buf[NUNA_MAX_PROBE_LINES];                   /* per sampled line: buffer, region,      */
     unsigned char line_region[NUNA_MAX_PROBE_LINES];                /* and the domain that reaches it faster  */
     unsigned char line_home[NUNA_MAX_PROBE_LINES];
+    /* Histograms of the per-(SM, line) hit latencies: bin b counts latencies in
+     * [NUNA_HIST_FIRST + b*NUNA_HIST_STEP, +NUNA_HIST_STEP) cycles; the last bin also takes everything above.
+     * hist_near: line at home in the SM's own domain; hist_far: in the other one (all pairs go to hist_near
+     * when the verdict is uniform).  The analogue of the paper's per-access latency distributions
+     * (Section 6.2).                                                                                     */
+    unsigned hist_near[NUNA_HIST_BINS];
+    unsigned hist_far[NUNA_HIST_BINS];
 } nuna_topology_t;
 
 /* Measures, for every SM (indexed by %smid) and every buffer, the latency of dependent L2-only loads
@@ -172,6 +182,18 @@ int nuna_plan_placement(const nuna_plan_input_t* in, int* m_compute, int* m_memo
  * call it explicitly before stream capture, because it allocates.  Growing the scratch later also
  * allocates.  Returns NUNA_ERR_CUDA if no device is usable.                                            */
 int nuna_init(size_t scratch_bytes);
+
+/* Tuning knobs of the current device's context (also read once from the environment variables of the
+ * same names, NUNA_BLOCKS etc., when the context is created).  value 0 restores the default.
+ *  NUNA_OPT_BLOCKS          cap on the grid size of every kernel (the paper's "number of thread blocks",
+ *                           Section 6.5: few blocks vs many)
+ *  NUNA_OPT_UNROLL          vectors per thread per work item (1, 2, 4; limited so that N * unroll <= 16)
+ *  NUNA_OPT_COLOC           destinations of a tile that share a block in the placement-aware one-shot (2, 4, 8)
+ *  NUNA_OPT_AUTO_MIN_BYTES  smallest message per rank for which NUNA_PLACE_AUTO may pick the aware kernel
+ *  NUNA_OPT_TIMEOUT_MS      flag-barrier timeout
+ * Returns NUNA_ERR_INVALID_ARG for an unknown option or a negative value.  Creates the context.          */
+enum { NUNA_OPT_BLOCKS = 0, NUNA_OPT_UNROLL = 1, NUNA_OPT_COLOC = 2, NUNA_OPT_AUTO_MIN_BYTES = 3, NUNA_OPT_TIMEOUT_MS = 4 };
+int nuna_set_option(int option, long long value);
 
 /* One-shot allreduce (Section 5.1, direct algorithm): every emulated rank d reads all N sources and
  * writes dst[d].  src[r], dst[d]: `count` elements each.  Work item = (tile, destination rank).       */

@@ -30,6 +30,8 @@ NUNA_PLACE_SM_LISTS = 128
 
 NUNA_MAX_SMS, NUNA_MAX_PROBE_BUFS, NUNA_PROBE_REGIONS, NUNA_MAX_PROBE_LINES = 256, 32, 8, 2048
 NUNA_TOPO_UNIFORM, NUNA_TOPO_NONUNIFORM = 0, 1
+NUNA_HIST_BINS, NUNA_HIST_FIRST, NUNA_HIST_STEP = 48, 200, 4
+NUNA_OPT_BLOCKS, NUNA_OPT_UNROLL, NUNA_OPT_COLOC, NUNA_OPT_AUTO_MIN_BYTES, NUNA_OPT_TIMEOUT_MS = 0, 1, 2, 3, 4
 
 
 class NunaTopology(ctypes.Structure):
@@ -51,6 +53,8 @@ class NunaTopology(ctypes.Structure):
         ("line_buf", ctypes.c_ubyte * NUNA_MAX_PROBE_LINES),
         ("line_region", ctypes.c_ubyte * NUNA_MAX_PROBE_LINES),
         ("line_home", ctypes.c_ubyte * NUNA_MAX_PROBE_LINES),
+        ("hist_near", ctypes.c_uint * NUNA_HIST_BINS),
+        ("hist_far", ctypes.c_uint * NUNA_HIST_BINS),
     ]
 
 
@@ -94,6 +98,8 @@ def lib() -> ctypes.CDLL:
         L.nuna_allreduce_twoshot_static.restype = ctypes.c_int
         L.nuna_allreduce_host.argtypes = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint, ctypes.c_int]
         L.nuna_allreduce_host.restype = ctypes.c_int
+        L.nuna_set_option.argtypes = [ctypes.c_int, ctypes.c_longlong]
+        L.nuna_set_option.restype = ctypes.c_int
         L.nuna_init.argtypes = [ctypes.c_size_t]
         L.nuna_init.restype = ctypes.c_int
         L.nuna_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
@@ -169,6 +175,10 @@ def _collective(name, src, dst, count, dtype, flags, stream, check, nranks=None)
 
 def nuna_init(scratch_bytes: int = 0, check: bool = True) -> int:
     return _finish(lib().nuna_init(scratch_bytes), "nuna_init", check)
+
+
+def nuna_set_option(option: int, value: int, check: bool = True) -> int:
+    return _finish(lib().nuna_set_option(option, value), "nuna_set_option", check)
 
 
 def nuna_allreduce_oneshot(src, dst, count, dtype=NUNA_BF16, flags=0, stream=None, check=True, nranks=None) -> int:

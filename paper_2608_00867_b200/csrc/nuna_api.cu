@@ -538,6 +538,24 @@ int nuna_init(size_t scratch_bytes)
     return ensure_scratch(c, scratch_bytes);
 }
 
+int nuna_set_option(int option, long long value)
+{
+    if (value < 0) return NUNA_ERR_INVALID_ARG;
+    Context* c = nullptr;
+    int st = get_context(&c);
+    if (st != NUNA_OK) return st;
+    std::lock_guard<std::mutex> lock(c->mutex);
+    switch (option) {
+        case NUNA_OPT_BLOCKS: c->blocks_override = (int)std::min<long long>(value, 1 << 22); break;
+        case NUNA_OPT_UNROLL: c->unroll_override = (int)value; break;
+        case NUNA_OPT_COLOC: c->coloc_override = (int)value; break;
+        case NUNA_OPT_AUTO_MIN_BYTES: c->auto_min_bytes = value ? (size_t)value : ((size_t)64 << 10); break;
+        case NUNA_OPT_TIMEOUT_MS: c->timeout_ns = (unsigned long long)(value ? value : 1000) * 1000000ull; break;
+        default: return NUNA_ERR_INVALID_ARG;
+    }
+    return NUNA_OK;
+}
+
 int nuna_allreduce_oneshot(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
                            unsigned flags, void* stream)
 {

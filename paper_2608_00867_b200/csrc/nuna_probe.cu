@@ -208,12 +208,24 @@ void analyse_topology(const std::vector<float>& lat, const std::vector<float>& l
             const double val = lat[(size_t)sms[i] * L + l];
             if (dom[i] == home[l]) { near_sum += val; ++near_n; } else { far_sum += val; ++far_n; }
         }
-    if (n1 == 0 || n1 == S || !near_n || !far_n) return;
+    auto bin_of = [](double cycles) {
+        int b = (int)std::floor((cycles - NUNA_HIST_FIRST) / NUNA_HIST_STEP);
+        return b < 0 ? 0 : (b >= NUNA_HIST_BINS ? NUNA_HIST_BINS - 1 : b);
+    };
+    const bool two_sided = !(n1 == 0 || n1 == S || !near_n || !far_n);
+    for (int i = 0; i < S; ++i)
+        for (int l = 0; l < L; ++l) {
+            const double val = lat[(size_t)sms[i] * L + l];
+            if (!two_sided || dom[i] == home[l]) out->hist_near[bin_of(val)]++; else out->hist_far[bin_of(val)]++;
+        }
+    if (!two_sided) return;
     out->near_lat = (float)(near_sum / near_n);
     out->far_lat = (float)(far_sum / far_n);
     out->domain_gap = out->far_lat - out->near_lat;
     for (int l = 0; l < L; ++l) out->line_home[l] = (unsigned char)home[l];
-    if (out->domain_gap > 3.0 * out->noise && out->domain_gap > 0.03 * median) {
+    if (!(out->domain_gap > 3.0 * out->noise && out->domain_gap > 0.03 * median)) {
+        for (int b = 0; b < NUNA_HIST_BINS; ++b) { out->hist_near[b] += out->hist_far[b]; out->hist_far[b] = 0; }
+    } else {
         out->verdict = NUNA_TOPO_NONUNIFORM;
         out->num_domains = 2;
         for (int i = 0; i < S; ++i) out->sm_domain[sms[i]] = dom[i];

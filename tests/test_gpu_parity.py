@@ -335,6 +335,30 @@ def test_sm_lists_replay_and_after_probe():
             assert_same_bits(got, want, "sm lists after probe")
 
 
+def test_tuning_options_change_the_launch_not_the_bits():
+    w = workloads.config_decode_activation()
+    src = workloads.special_values(w.nranks, w.count + 5, seed=44)
+    want = oracle.allreduce(src, nthreads=4)[0]
+    dsrc = upload(src)
+    try:
+        for opt, values in ((nb.NUNA_OPT_BLOCKS, (1, 7, 148, 100000)), (nb.NUNA_OPT_UNROLL, (1, 2, 4)),
+                            (nb.NUNA_OPT_COLOC, (2, 4, 8))):
+            for v in values:
+                nb.nuna_set_option(opt, v)
+                for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE),
+                                    (nb.nuna_allreduce_twoshot, 0), (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
+                    dst = Dst(w.nranks, w.count + 5)
+                    call(dsrc, dst.view, w.count + 5, flags=flags)
+                    assert_same_bits(dst.numpy()[w.nranks - 1], want, f"option {opt}={v} {call.__name__} {flags}")
+            nb.nuna_set_option(opt, 0)
+        assert nb.nuna_set_option(99, 1, check=False) == nb.NUNA_ERR_INVALID_ARG
+        assert nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, -1, check=False) == nb.NUNA_ERR_INVALID_ARG
+    finally:
+        for opt in (nb.NUNA_OPT_BLOCKS, nb.NUNA_OPT_UNROLL, nb.NUNA_OPT_COLOC):
+            nb.nuna_set_option(opt, 0)
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
 def test_host_buffer_entry_point():
     for n, count, two in ((8, 32 * 8192, False), (8, 32 * 8192, True), (3, 1001, False), (3, 1001, True)):
         src = workloads.rank_buffers(n, count, "normal", seed=77)

@@ -50,6 +50,7 @@ def test_uniform_matrix_gives_uniform_verdict():
     t = nb.debug_analyse_topology(a, b)
     assert t.verdict == nb.NUNA_TOPO_UNIFORM and t.num_domains == 1
     assert all(d == 0 for d in t.sm_domain[:148])
+    assert sum(t.hist_near[:]) == 148 * 300 and sum(t.hist_far[:]) == 0
 
 
 def test_two_clusters_are_recovered_exactly():
@@ -61,6 +62,10 @@ def test_two_clusters_are_recovered_exactly():
     assert np.array_equal(got, dom)                         # SM 0 is in domain 0 by construction
     assert np.array_equal(np.array(t.line_home[:400]), home)
     assert 27.0 < t.domain_gap < 33.0
+    near, far = np.array(t.hist_near[:]), np.array(t.hist_far[:])
+    assert near.sum() + far.sum() == 148 * 400 and near.sum() > 0 and far.sum() > 0
+    centre = lambda h: (h * (nb.NUNA_HIST_FIRST + nb.NUNA_HIST_STEP * (np.arange(len(h)) + 0.5))).sum() / h.sum()
+    assert 25.0 < centre(far) - centre(near) < 35.0          # the histograms show the same gap
     assert 0.5 < t.noise < 2.5
     assert t.far_lat > t.near_lat
 
