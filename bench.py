@@ -210,6 +210,24 @@ def run_gpu(args):
         del g
         return ms * 1e3 / (nodes * replays)
 
+    def per_call_stats(fn, sets, nodes, replays):
+        """Each replay of the graph timed on its own (its own event pair): median / min / max per call."""
+        g = capture(fn, sets, nodes)
+        with torch.cuda.stream(stream):
+            g.replay()
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(replays + 1)]
+            barrier()
+            t0 = time.time()
+            evs[0].record(stream)
+            for i in range(replays):
+                g.replay()
+                evs[i + 1].record(stream)
+            barrier()
+            sampler.mark(t0, time.time())
+        per = sorted(max_over_ranks(evs[i].elapsed_time(evs[i + 1])) * 1e3 / nodes for i in range(replays))
+        del g
+        return {"median": per[len(per) // 2], "min": per[0], "max": per[-1]}
+
     # ---- headline: K one-shot allreduces on the decode activation ------------------------------------
     w = workloads.config_decode_activation()
     count = w.count
@@ -351,12 +369,15 @@ def run_gpu(args):
             c, B = wl.count, wl.bytes_per_rank
             ssets = make_sets(N_RANKS, c, c, 2 * l2 + (64 << 20), "normal", wl.seed)
             nodes_s = max(len(ssets), min(512, (256 << 20) // B + 1))          # at least one full rotation
-            reps = 3 if B <= (4 << 20) else 2
-            row = {"bytes_per_rank": B, "buffer_sets": len(ssets), "algorithmic_bytes": 2 * N_RANKS * B}
+            reps = 7 if B <= (4 << 20) else 5
+            row = {"bytes_per_rank": B, "buffer_sets": len(ssets), "algorithmic_bytes": 2 * N_RANKS * B,
+                   "calls_per_sample": nodes_s, "samples": reps}
             for name, mk in algos.items():
-                cold = per_call_us(mk(c), ssets, nodes_s, reps)
-                warm = per_call_us(mk(c), ssets[:1], nodes_s, reps)
-                row[name] = {"cold_us": round(cold, 3), "warm_us": round(warm, 3),
+                cs = per_call_stats(mk(c), ssets, nodes_s, reps)
+                warm = per_call_stats(mk(c), ssets[:1], nodes_s, reps)["median"]
+                cold = cs["median"]
+                row[name] = {"cold_us": round(cold, 3), "cold_min_us": round(cs["min"], 3), "cold_max_us": round(cs["max"], 3),
+                             "warm_us": round(warm, 3),
                              "cold_gbs": round(2 * N_RANKS * B / cold / 1e3, 1),
                              "cold_frac_of_peak": round(2 * N_RANKS * B / cold / 1e3 / peak_gbs, 4)}
             best = min(algos, key=lambda a: row[a]["cold_us"])

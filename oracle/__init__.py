@@ -47,6 +47,15 @@ def _load():
             fn = getattr(lib, name)
             fn.argtypes = [pp, pp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int]
             fn.restype = None
+        for name in ("nuna_oracle_allreduce_f16", "nuna_oracle_allreduce_f32",
+                     "nuna_oracle_reduce_scatter_f16", "nuna_oracle_reduce_scatter_f32"):
+            fn = getattr(lib, name)
+            fn.argtypes = [pp, pp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int]
+            fn.restype = None
+        lib.nuna_oracle_rne_f16.argtypes = [ctypes.c_float]
+        lib.nuna_oracle_rne_f16.restype = ctypes.c_uint16
+        lib.nuna_oracle_widen_f16.argtypes = [ctypes.c_uint16]
+        lib.nuna_oracle_widen_f16.restype = ctypes.c_float
         lib.nuna_oracle_fold_bf16.argtypes = [ctypes.c_void_p, ctypes.c_int]
         lib.nuna_oracle_fold_bf16.restype = ctypes.c_uint16
         lib.nuna_oracle_rne_bf16.argtypes = [ctypes.c_float]
@@ -57,42 +66,46 @@ def _load():
     return _lib
 
 
+# Element types.  Buffers are raw bit patterns: uint16 for bf16 / f16, uint32 for f32.
+STORAGE = {"bf16": np.uint16, "f16": np.uint16, "f32": np.uint32}
+
+
 def _ptrs(arrs: Sequence[np.ndarray]):
     tab = (ctypes.c_void_p * len(arrs))()
     for i, a in enumerate(arrs):
-        assert a.dtype == np.uint16 and a.flags.c_contiguous
+        assert a.dtype in (np.uint16, np.uint32) and a.flags.c_contiguous
         tab[i] = a.ctypes.data
     return tab
 
 
-def _check_src(src: Sequence[np.ndarray], length: int):
+def _check_src(src: Sequence[np.ndarray], length: int, storage=np.uint16):
     if len(src) < 1:
         raise ValueError("need at least one rank")
     for a in src:
-        if a.dtype != np.uint16 or a.ndim != 1 or len(a) != length:
-            raise ValueError("every rank buffer must be a 1-D uint16 array of the same length")
+        if a.dtype != storage or a.ndim != 1 or len(a) != length:
+            raise ValueError(f"every rank buffer must be a 1-D {np.dtype(storage).name} array of the same length")
 
 
-def allreduce(src: Sequence[np.ndarray], nthreads: int = 1) -> List[np.ndarray]:
+def allreduce(src: Sequence[np.ndarray], nthreads: int = 1, dtype: str = "bf16") -> List[np.ndarray]:
     """One result array per destination rank (all equal by definition)."""
     n, count = len(src), len(src[0])
-    _check_src(src, count)
+    _check_src(src, count, STORAGE[dtype])
     src = [np.ascontiguousarray(a) for a in src]
-    dst = [np.empty(count, dtype=np.uint16) for _ in range(n)]
-    _load().nuna_oracle_allreduce_bf16(_ptrs(src), _ptrs(dst), n, count, int(nthreads))
+    dst = [np.empty(count, dtype=STORAGE[dtype]) for _ in range(n)]
+    getattr(_load(), f"nuna_oracle_allreduce_{dtype}")(_ptrs(src), _ptrs(dst), n, count, int(nthreads))
     return dst
 
 
-def reduce_scatter(src: Sequence[np.ndarray], nthreads: int = 1) -> List[np.ndarray]:
+def reduce_scatter(src: Sequence[np.ndarray], nthreads: int = 1, dtype: str = "bf16") -> List[np.ndarray]:
     """``src[k]`` holds ``N*S`` elements; returns N arrays of S elements."""
     n, total = len(src), len(src[0])
-    _check_src(src, total)
+    _check_src(src, total, STORAGE[dtype])
     if total % n:
         raise ValueError("source length must be a multiple of the rank count")
     shard = total // n
     src = [np.ascontiguousarray(a) for a in src]
-    dst = [np.empty(shard, dtype=np.uint16) for _ in range(n)]
-    _load().nuna_oracle_reduce_scatter_bf16(_ptrs(src), _ptrs(dst), n, shard, int(nthreads))
+    dst = [np.empty(shard, dtype=STORAGE[dtype]) for _ in range(n)]
+    getattr(_load(), f"nuna_oracle_reduce_scatter_{dtype}")(_ptrs(src), _ptrs(dst), n, shard, int(nthreads))
     return dst
 
 
@@ -122,6 +135,14 @@ def fold(vals) -> int:
     """Rank-ordered sum of one column of bf16 patterns."""
     a = np.ascontiguousarray(np.asarray(vals, dtype=np.uint16))
     return int(_load().nuna_oracle_fold_bf16(a.ctypes.data, len(a)))
+
+
+def rne_f16(x: float) -> int:
+    return int(_load().nuna_oracle_rne_f16(x))
+
+
+def widen_f16(h: int) -> float:
+    return float(_load().nuna_oracle_widen_f16(h))
 
 
 def rne_bf16(x: float) -> int:

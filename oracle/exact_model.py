@@ -98,6 +98,78 @@ def encode_bf16(v: Value) -> int:
     return (sign << 15) | ((e + 127) << 7) | int(m.numerator)
 
 
+# ---- the same model for binary16 and binary32 storage ----------------------------------------------------
+
+_FORMATS = {            # name: (exponent bits, fraction bits)
+    "bf16": (8, 7), "f16": (5, 10), "f32": (8, 23),
+}
+
+
+def decode(h: int, fmt: str) -> Value:
+    ebits, fbits = _FORMATS[fmt]
+    bias = (1 << (ebits - 1)) - 1
+    sign = (h >> (ebits + fbits)) & 1
+    expo = (h >> fbits) & ((1 << ebits) - 1)
+    mant = h & ((1 << fbits) - 1)
+    if expo == (1 << ebits) - 1:
+        return ("inf", sign) if mant == 0 else ("nan",)
+    if expo == 0:
+        return ("fin", sign, Fraction(mant, 1 << fbits) * Fraction(2) ** (1 - bias))
+    return ("fin", sign, (1 + Fraction(mant, 1 << fbits)) * Fraction(2) ** (expo - bias))
+
+
+def _round_mag_fmt(mag: Fraction, precision: int, emin: int, emax: int):
+    if mag == 0:
+        return mag
+    e = max(_floor_log2(mag), emin)
+    quantum = Fraction(2) ** (e - precision + 1)
+    q = mag / quantum
+    n = q.numerator // q.denominator
+    rem = q - n
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and n % 2 == 1):
+        n += 1
+    out = n * quantum
+    return None if out >= Fraction(2) ** (emax + 1) else out
+
+
+def encode(v: Value, fmt: str) -> int:
+    ebits, fbits = _FORMATS[fmt]
+    bias = (1 << (ebits - 1)) - 1
+    top = ((1 << ebits) - 1) << fbits
+    sbit = ebits + fbits
+    if v[0] == "nan":
+        return (1 << sbit) - 1                      # canonical: all ones below the sign bit
+    if v[0] == "inf":
+        return (v[1] << sbit) | top
+    sign = v[1]
+    mag = _round_mag_fmt(v[2], fbits + 1, 1 - bias, bias)
+    if mag is None:
+        return (sign << sbit) | top
+    if mag == 0:
+        return sign << sbit
+    e = _floor_log2(mag)
+    if e < 1 - bias:
+        m = mag / Fraction(2) ** (1 - bias - fbits)
+        assert m.denominator == 1
+        return (sign << sbit) | int(m.numerator)
+    m = (mag / Fraction(2) ** e - 1) * (1 << fbits)
+    assert m.denominator == 1
+    return (sign << sbit) | ((e + bias) << fbits) | int(m.numerator)
+
+
+def fold_fmt(column: Sequence[int], fmt: str) -> int:
+    """Left fold with binary32 partial sums over values stored in `fmt`, then one round to `fmt`."""
+    acc = decode(int(column[0]), fmt)
+    for h in column[1:]:
+        acc = add_binary32(acc, decode(int(h), fmt))
+    return encode(acc, fmt)
+
+
+def is_nan_fmt(h: int, fmt: str) -> bool:
+    ebits, fbits = _FORMATS[fmt]
+    return ((h >> fbits) & ((1 << ebits) - 1)) == (1 << ebits) - 1 and (h & ((1 << fbits) - 1)) != 0
+
+
 def fold(column: Sequence[int]) -> int:
     """Left fold in rank order with binary32 partial sums, then one round to bf16."""
     acc = decode_bf16(int(column[0]))

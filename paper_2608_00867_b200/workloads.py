@@ -103,24 +103,48 @@ CHAIN_TOKENS = (1, 8, 64, 256)
 
 # ---- adversarial value mixes for parity (not benchmark inputs) --------------------------
 
-def special_values(nranks: int, count: int, seed: int) -> List[np.ndarray]:
-    """Random 16-bit patterns biased towards the awkward corners of bf16.
+def special_values(nranks: int, count: int, seed: int, dtype: str = "bf16") -> List[np.ndarray]:
+    """Random bit patterns biased towards the awkward corners of the element type.
 
     A third of the elements are arbitrary bit patterns (NaN, Inf, subnormals
     included), a third are small integers whose sums are exact, the rest are
     values with mantissa ties around 1.0 so that round-to-nearest-even matters.
+    Returned as raw storage words: uint16 for bf16 / f16, uint32 for f32.
     """
     rng = np.random.Generator(np.random.PCG64(seed))
+    tdt = {"bf16": torch.bfloat16, "f16": torch.float16, "f32": torch.float32}[dtype]
+    if dtype == "f32":
+        word, view, bits = np.uint32, torch.int32, 32
+        one, tiny = 0x3F800000, 0x33800000            # 1.0 and 2^-24 (half an ulp of 1.0)
+    elif dtype == "f16":
+        word, view, bits = np.uint16, torch.int16, 16
+        one, tiny = 0x3C00, 0x1000                    # 1.0 and 2^-11
+    else:
+        word, view, bits = np.uint16, torch.int16, 16
+        one, tiny = 0x3F80, 0x3B80                    # 1.0 and 2^-8
     out = []
     for _ in range(nranks):
         kind = rng.integers(0, 3, size=count)
-        raw = rng.integers(0, 1 << 16, size=count, dtype=np.uint32).astype(np.uint16)
+        raw = rng.integers(0, 1 << bits, size=count, dtype=np.uint64).astype(word)
         ints = torch.from_numpy(rng.integers(-8, 9, size=count).astype(np.float32)) \
-            .to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
-        # 1.0 + k*2^-7 and k*2^-8: sums of these land on bf16 rounding ties
+            .to(tdt).view(view).numpy().view(word)
+        # 1.0 + k ulp and +-(half an ulp of 1.0): sums of these land on rounding ties
         ties = np.where(rng.integers(0, 2, size=count) == 0,
-                        (0x3F80 + rng.integers(0, 4, size=count)).astype(np.uint16),
-                        (0x3B80 + rng.integers(0, 2, size=count) * 0x8000).astype(np.uint16))
-        buf = np.where(kind == 0, raw, np.where(kind == 1, ints, ties)).astype(np.uint16)
+                        (one + rng.integers(0, 4, size=count)).astype(word),
+                        (tiny + rng.integers(0, 2, size=count) * (1 << (bits - 1))).astype(word))
+        buf = np.where(kind == 0, raw, np.where(kind == 1, ints, ties)).astype(word)
         out.append(buf)
+    return out
+
+
+def rank_buffers_typed(nranks: int, count: int, dist: str, seed: int, dtype: str) -> List[np.ndarray]:
+    """Like rank_buffers, for any element type (raw storage words)."""
+    tdt = {"bf16": torch.bfloat16, "f16": torch.float16, "f32": torch.float32}[dtype]
+    view, word = (torch.int32, np.uint32) if dtype == "f32" else (torch.int16, np.uint16)
+    out = []
+    for r in range(nranks):
+        gen = torch.Generator(device="cpu")
+        gen.manual_seed((int(seed) << 20) + r)
+        x = torch.randn(count, generator=gen) if dist == "normal" else torch.rand(count, generator=gen) * 2.0 - 1.0
+        out.append(x.to(tdt).view(view).numpy().view(word).copy())
     return out

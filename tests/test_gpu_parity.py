@@ -173,7 +173,7 @@ def test_sweep_sizes_one_and_two_shot_agree_with_oracle():
 
 
 def test_full_size_64MiB_sampled_columns_and_invariants():
-    """BASELINE's largest point, in the launch configuration the benchmark times."""
+    """The largest benchmarked message (8 ranks x 64 MiB), in the launch configuration the benchmark times."""
     w = workloads.config_size_sweep(26, 26)[0]
     n, count = w.nranks, w.count
     gen = torch.Generator(device="cuda")
