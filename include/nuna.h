@@ -10,11 +10,14 @@
  * with the latency-optimised direct / all-pairs algorithm (Section 5.1), and
  * the thread-block placement idea of Section 4.2 (Algorithm 1) mapped onto SMs.
  *
- * Numerics (bf16): dst = rne_bf16((((f(src[0]) + f(src[1])) + ...) + f(src[N-1])))
- * with every partial sum an IEEE binary32 (round to nearest even, subnormals
- * kept), ranks folded in the fixed order 0..N-1 starting from rank 0's value,
- * and ONE final round-to-nearest-even to bf16.  A NaN result is the canonical
- * 0x7FFF.  Every destination receives the same bits.  Allgather is a bit copy.
+ * Numerics: dst = rne_T((((f(src[0]) + f(src[1])) + ...) + f(src[N-1]))) where f
+ * widens the storage type T exactly to binary32, every partial sum is an IEEE
+ * binary32 (round to nearest even, subnormals kept), ranks are folded in the
+ * fixed order 0..N-1 starting from rank 0's value, and there is ONE final
+ * round-to-nearest-even to T (none for T = binary32).  T is bf16 (the type the
+ * benchmarks use), IEEE binary16 or binary32.  A NaN result is canonical
+ * (0x7FFF / 0x7FFFFFFF).  Every destination receives the same bits.  Allgather
+ * and alltoall are bit copies.
  *
  * Conventions, all entry points:
  *  - `src` / `dst` are HOST arrays of `nranks` DEVICE pointers (except in
@@ -57,7 +60,7 @@ typedef enum {
     NUNA_ERR_TOO_LARGE = 9
 } nuna_status_t;
 
-typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* only NUNA_BF16 is implemented */
+typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* element (storage) type; 2, 2, 4 bytes */
 
 #define NUNA_MAX_RANKS 16
 
@@ -203,7 +206,7 @@ int nuna_allreduce_oneshot(const void* const* src, void* const* dst, int nranks,
 /* Two-shot allreduce: reduce-scatter over N contiguous chunks (emulated rank r reduces chunk r), an
  * in-kernel flag barrier among the persistent thread blocks, then a put-style allgather of the chunks
  * into every destination.  Same bits as the one-shot.  Any `count`; chunk = ceil(count/N) rounded up
- * to 8 elements, trailing chunks may be short or empty.  Uses the context's shard scratch
+ * to a whole 16-byte vector, trailing chunks may be short or empty.  Uses the context's shard scratch
  * (count*elemsize bytes, grown on demand) unless NUNA_TWOSHOT_PUT is set.  Calls that share the
  * context must be stream-ordered with respect to each other.                                          */
 int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
@@ -235,9 +238,9 @@ int nuna_alltoall(const void* const* src, void* const* dst, int nranks,
  * exactly what nuna_allreduce_twoshot computes (flag-barrier form, same bits) but takes its shard
  * intermediate and its barrier words from a fixed array compiled into the library, so it never calls
  * cudaMalloc, cudaFree or any allocating routine, and it does not create the per-device context.
- *  - Limit: count <= NUNA_STATIC_MAX_COUNT elements per rank (4 MiB of bf16); larger counts return
- *    NUNA_ERR_TOO_LARGE and print the limit.  The array costs 4 MiB of device memory on every GPU
- *    that loads the library, for the life of the process.
+ *  - Limit: 4 MiB per rank, i.e. count <= NUNA_STATIC_MAX_COUNT elements of a 16-bit type (half that
+ *    many of binary32); larger messages return NUNA_ERR_TOO_LARGE and print the limit.  The array
+ *    costs 4 MiB of device memory on every GPU that loads the library, for the life of the process.
  *  - The first call on a device looks up the array's device address and zeroes the barrier words
  *    (a synchronous 16-byte cudaMemset); make that first call before starting any stream capture.
  *  - All calls on a device share the one array, which keeps the previous call's shard; the kernel

@@ -21,6 +21,8 @@ NUNA_ERR_TOO_MANY_RANKS = 8
 NUNA_ERR_TOO_LARGE = 9
 
 NUNA_BF16, NUNA_F16, NUNA_F32 = 0, 1, 2
+DTYPE_BY_NAME = {"bf16": NUNA_BF16, "f16": NUNA_F16, "f32": NUNA_F32}
+ELEM_SIZE = {NUNA_BF16: 2, NUNA_F16: 2, NUNA_F32: 4}
 NUNA_MAX_RANKS = 16
 NUNA_PLACE_ROUNDROBIN, NUNA_PLACE_AWARE, NUNA_PLACE_AUTO = 0, 1, 2
 NUNA_TWOSHOT_PUT = 16

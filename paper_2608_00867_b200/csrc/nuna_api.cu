@@ -68,6 +68,9 @@ int ensure_scratch(Context* c, size_t bytes)
 
 // ---- argument validation -------------------------------------------------------------------
 
+size_t elem_size(int dtype) { return dtype == NUNA_F32 ? 4 : 2; }
+static size_t elems_per_vec(int dtype) { return 16 / elem_size(dtype); }
+
 static bool overlaps(const void* a, size_t na, const void* b, size_t nb)
 {
     const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
@@ -79,8 +82,7 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
 {
     if (nranks > NUNA_MAX_RANKS) return NUNA_ERR_TOO_MANY_RANKS;
     if (nranks < 1) return NUNA_ERR_INVALID_ARG;
-    if (dtype != NUNA_BF16) return (dtype == NUNA_F16 || dtype == NUNA_F32) ? NUNA_ERR_UNSUPPORTED_DTYPE
-                                                                             : NUNA_ERR_UNSUPPORTED_DTYPE;
+    if (dtype != NUNA_BF16 && dtype != NUNA_F16 && dtype != NUNA_F32) return NUNA_ERR_UNSUPPORTED_DTYPE;
     if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT | NUNA_HINT_RESIDENT | NUNA_LAUNCH_PDL | NUNA_PLACE_SM_LISTS)) != 0u ||
         (flags & NUNA_PLACE_MASK) == 3u)
         return NUNA_ERR_INVALID_ARG;
@@ -91,7 +93,7 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
         if (!src[r] || !dst[r]) return NUNA_ERR_INVALID_ARG;
         if (device_ptrs && (((uintptr_t)src[r] | (uintptr_t)dst[r]) & 15u)) return NUNA_ERR_ALIGNMENT;
     }
-    const size_t sb = src_elems * 2, db = dst_elems * 2;
+    const size_t sb = src_elems * elem_size(dtype), db = dst_elems * elem_size(dtype);
     for (int d = 0; d < nranks; ++d) {
         for (int r = 0; r < nranks; ++r)
             if (overlaps(dst[d], db, src[r], sb)) return NUNA_ERR_ALIAS;
@@ -191,30 +193,42 @@ static int launch(void (*kernel)(Args...), unsigned grid, cudaStream_t stream, u
 // Compile-time dispatch over the rank count N and the unroll factor U (N * U <= 16 vectors in flight).
 template <int V> using IC = std::integral_constant<int, V>;
 
-template <int N, typename F>
-static int dispatch_u(int u, F&& f)
+template <int N, int U, typename F>
+static int dispatch_dt(int dtype, F&& f)
 {
-    if constexpr (N * 4 <= 16) { if (u == 4) return f(IC<N>{}, IC<4>{}); }
-    if constexpr (N * 2 <= 16) { if (u >= 2) return f(IC<N>{}, IC<2>{}); }
-    return f(IC<N>{}, IC<1>{});
+    switch (dtype) {
+        case NUNA_BF16: return f(IC<N>{}, IC<U>{}, IC<kBf16>{});
+        case NUNA_F16: return f(IC<N>{}, IC<U>{}, IC<kF16>{});
+        case NUNA_F32: return f(IC<N>{}, IC<U>{}, IC<kF32>{});
+        default: return NUNA_ERR_UNSUPPORTED_DTYPE;
+    }
+}
+
+template <int N, typename F>
+static int dispatch_u(int u, int dtype, F&& f)
+{
+    if constexpr (N * 4 <= 16) { if (u == 4) return dispatch_dt<N, 4>(dtype, f); }
+    if constexpr (N * 2 <= 16) { if (u >= 2) return dispatch_dt<N, 2>(dtype, f); }
+    return dispatch_dt<N, 1>(dtype, f);
 }
 
 template <typename F>
-static int dispatch(int nranks, int u, F&& f)
+static int dispatch(int nranks, int u, int dtype, F&& f)
 {
     switch (nranks) {
-        case 1: return dispatch_u<1>(u, f);   case 2: return dispatch_u<2>(u, f);
-        case 3: return dispatch_u<3>(u, f);   case 4: return dispatch_u<4>(u, f);
-        case 5: return dispatch_u<5>(u, f);   case 6: return dispatch_u<6>(u, f);
-        case 7: return dispatch_u<7>(u, f);   case 8: return dispatch_u<8>(u, f);
-        case 9: return dispatch_u<9>(u, f);   case 10: return dispatch_u<10>(u, f);
-        case 11: return dispatch_u<11>(u, f); case 12: return dispatch_u<12>(u, f);
-        case 13: return dispatch_u<13>(u, f); case 14: return dispatch_u<14>(u, f);
-        case 15: return dispatch_u<15>(u, f); case 16: return dispatch_u<16>(u, f);
+        case 1: return dispatch_u<1>(u, dtype, f);   case 2: return dispatch_u<2>(u, dtype, f);
+        case 3: return dispatch_u<3>(u, dtype, f);   case 4: return dispatch_u<4>(u, dtype, f);
+        case 5: return dispatch_u<5>(u, dtype, f);   case 6: return dispatch_u<6>(u, dtype, f);
+        case 7: return dispatch_u<7>(u, dtype, f);   case 8: return dispatch_u<8>(u, dtype, f);
+        case 9: return dispatch_u<9>(u, dtype, f);   case 10: return dispatch_u<10>(u, dtype, f);
+        case 11: return dispatch_u<11>(u, dtype, f); case 12: return dispatch_u<12>(u, dtype, f);
+        case 13: return dispatch_u<13>(u, dtype, f); case 14: return dispatch_u<14>(u, dtype, f);
+        case 15: return dispatch_u<15>(u, dtype, f); case 16: return dispatch_u<16>(u, dtype, f);
         default: return NUNA_ERR_TOO_MANY_RANKS;
     }
 }
-#define NUNA_NU(n_, u_) constexpr int N = decltype(n_)::value; constexpr int U = decltype(u_)::value; (void)U
+#define NUNA_NUD(n_, u_, d_) constexpr int N = decltype(n_)::value; constexpr int U = decltype(u_)::value; \
+    constexpr int DT = decltype(d_)::value; (void)U; (void)DT
 
 static size_t ceil_div(size_t a, size_t b) { return (a + b - 1) / b; }
 
@@ -222,10 +236,9 @@ static size_t ceil_div(size_t a, size_t b) { return (a + b - 1) / b; }
 
 // NUNA_PLACE_AUTO: use the placement-aware kernel only where it is at least as fast as the
 // round-robin baseline.  NUNA_AUTO_MIN_BYTES overrides the measured crossover (bytes per rank).
-static bool aware_pays_off(const Context* c, int nranks, size_t count, unsigned flags)
+static bool aware_pays_off(const Context* c, int nranks, size_t bytes, unsigned flags)
 {
     if (nranks < 2 || !(flags & NUNA_HINT_RESIDENT)) return false;
-    const size_t bytes = count * 2;
     // sources and destinations of one call, twice over (the producer's other buffers), must fit in L2
     // for "resident" to be physically possible
     if (4 * bytes * (size_t)nranks > c->l2_bytes) return false;
@@ -308,17 +321,17 @@ void plan_oneshot_lists(const nuna_topology_t* topo, int num_sms, int nranks, si
     }
 }
 
-static int get_sm_plan(Context* c, int nranks, size_t count, int coloc, cudaStream_t stream, SmPlan** out)
+static int get_sm_plan(Context* c, int nranks, size_t nvec, int coloc, cudaStream_t stream, SmPlan** out)
 {
     std::lock_guard<std::mutex> lock(c->mutex);
-    const auto key = std::make_tuple(nranks, count, coloc);
+    const auto key = std::make_tuple(nranks, nvec, coloc);
     auto it = c->sm_plans.find(key);
     if (it == c->sm_plans.end()) {
         cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
         if (cudaStreamIsCapturing(stream, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone)
             return NUNA_ERR_CAPTURING;                 // building a plan allocates: make one plain call first
         const size_t lanes = (size_t)(kThreads / coloc);
-        const size_t ntiles = ceil_div(count / kVecElems, lanes);
+        const size_t ntiles = ceil_div(nvec, lanes);
         std::vector<std::vector<unsigned>> lists;
         plan_oneshot_lists(c->have_topology ? &c->topology : nullptr, c->num_sms, nranks, ntiles, lanes * 16,
                            ntiles <= kGenericPlanTiles, lists);
@@ -363,22 +376,22 @@ static int coloc_for(const Context* c, int nranks)
 }
 
 // Everything a later launch of this shape would have to allocate (called before stream capture).
-int prepare_oneshot(Context* c, int nranks, size_t count, unsigned flags)
+int prepare_oneshot(Context* c, int nranks, int dtype, size_t count, unsigned flags)
 {
     if ((flags & NUNA_PLACE_MASK) == NUNA_PLACE_AWARE && (flags & NUNA_PLACE_SM_LISTS)) {
         SmPlan* pl = nullptr;
-        return get_sm_plan(c, nranks, count, coloc_for(c, nranks), (cudaStream_t)0, &pl);
+        return get_sm_plan(c, nranks, count / elems_per_vec(dtype), coloc_for(c, nranks), (cudaStream_t)0, &pl);
     }
     return NUNA_OK;
 }
 
-template <int N, int C>
+template <int N, int C, int DT>
 static int launch_sm_lists(Context* c, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
 {
     static int occ = 0;
-    auto k = k_oneshot_sm<N, C>;
+    auto k = k_oneshot_sm<N, C, DT>;
     SmPlan* pl = nullptr;
-    const int st = get_sm_plan(c, N, count, C, stream, &pl);
+    const int st = get_sm_plan(c, N, count / Elem<DT>::kElems, C, stream, &pl);
     if (st != NUNA_OK) return st;
     SmLists sl;
     sl.off = pl->off; sl.tiles = pl->tiles; sl.cursor = pl->cursor; sl.present = pl->present; sl.ctl = pl->ctl;
@@ -389,112 +402,129 @@ static int launch_sm_lists(Context* c, const RankPtrs& p, size_t count, unsigned
     return launch(k, grid, stream, mode, p, count, sl, blocks_per_sm);
 }
 
-template <int N, int C>
+template <int N, int C, int DT>
 static int launch_group(Context* c, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
 {
     static int occ = 0;
-    auto k = k_oneshot_group<N, C>;
-    const size_t nvec = count / kVecElems;
+    auto k = k_oneshot_group<N, C, DT>;
+    const size_t nvec = count / Elem<DT>::kElems;
     const size_t ntiles = ceil_div(nvec, (size_t)(kThreads / C));
-    const size_t nitems = std::max<size_t>(ntiles * ((N + C - 1) / C), (count % kVecElems) ? (size_t)N : 0);
+    const size_t nitems = std::max<size_t>(ntiles * ((N + C - 1) / C), (count % Elem<DT>::kElems) ? (size_t)N : 0);
     const unsigned grid = pick_grid(c, nitems, occupancy(c, k, &occ));
     return launch(k, grid, stream, mode, p, count, ntiles);
 }
 
-int launch_oneshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream)
+int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t count, unsigned flags, cudaStream_t stream)
 {
-    const unsigned mode = launch_mode(flags, count * 2 * (size_t)nranks);
-    const size_t nvec = count / kVecElems;
+    const size_t bytes = count * elem_size(dtype);                   // per rank
+    const size_t epv = elems_per_vec(dtype);
+    const unsigned mode = launch_mode(flags, bytes * (size_t)nranks);
+    const size_t nvec = count / epv;
     const unsigned place = flags & NUNA_PLACE_MASK;
-    if (place == NUNA_PLACE_AWARE || (place == NUNA_PLACE_AUTO && aware_pays_off(c, nranks, count, flags))) {
+    if (place == NUNA_PLACE_AWARE || (place == NUNA_PLACE_AUTO && aware_pays_off(c, nranks, bytes, flags))) {
         // co-location factor: C destinations of a tile share a block (C <= N rounded up to a power of two)
         const int coloc = coloc_for(c, nranks);
         if (flags & NUNA_PLACE_SM_LISTS) {
-            return dispatch(nranks, 1, [&](auto n_, auto) -> int {
-                constexpr int N = decltype(n_)::value;
-                if (coloc >= 8) return launch_sm_lists<N, 8>(c, p, count, mode, stream);
-                if (coloc >= 4) return launch_sm_lists<N, 4>(c, p, count, mode, stream);
-                return launch_sm_lists<N, 2>(c, p, count, mode, stream);
+            return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
+                constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
+                if (coloc >= 8) return launch_sm_lists<N, 8, DT>(c, p, count, mode, stream);
+                if (coloc >= 4) return launch_sm_lists<N, 4, DT>(c, p, count, mode, stream);
+                return launch_sm_lists<N, 2, DT>(c, p, count, mode, stream);
             });
         }
-        return dispatch(nranks, 1, [&](auto n_, auto) -> int {
-            constexpr int N = decltype(n_)::value;
-            if (coloc >= 8) return launch_group<N, 8>(c, p, count, mode, stream);
-            if (coloc >= 4) return launch_group<N, 4>(c, p, count, mode, stream);
-            return launch_group<N, 2>(c, p, count, mode, stream);
+        return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
+            constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
+            if (coloc >= 8) return launch_group<N, 8, DT>(c, p, count, mode, stream);
+            if (coloc >= 4) return launch_group<N, 4, DT>(c, p, count, mode, stream);
+            return launch_group<N, 2, DT>(c, p, count, mode, stream);
         });
     }
-    return dispatch(nranks, pick_unroll(c, nranks), [&](auto n_, auto u_) -> int {
-        NUNA_NU(n_, u_);
+    return dispatch(nranks, pick_unroll(c, nranks), dtype, [&](auto n_, auto u_, auto d_) -> int {
+        NUNA_NUD(n_, u_, d_);
         static int occ = 0;
-        auto k = k_oneshot_rr<N, U>;
+        auto k = k_oneshot_rr<N, U, DT>;
         const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
-        const size_t nitems = std::max<size_t>(ntiles * N, (count % kVecElems) ? (size_t)N : 0);
+        const size_t nitems = std::max<size_t>(ntiles * N, (count % epv) ? (size_t)N : 0);
         // one resident wave while the message is small enough for latency to matter, four beyond
-        const unsigned grid = pick_grid(c, nitems, occupancy(c, k, &occ), count * 2 >= ((size_t)8 << 20) ? 4 : 1);
+        const unsigned grid = pick_grid(c, nitems, occupancy(c, k, &occ), bytes >= ((size_t)8 << 20) ? 4 : 1);
         return launch(k, grid, stream, mode, p, count, ntiles);
     });
 }
 
-int launch_twoshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream)
+// Launches the flag-barrier two-shot on explicit scratch / barrier storage (the context's, or the
+// fixed arrays of the allocation-free entry point).
+static int launch_twoshot_fused(int num_sms, int blocks_override, const RankPtrs& p, int nranks, int dtype, size_t count,
+                                int u, uint4* scratch, BarrierWords* bw, unsigned long long timeout_ns,
+                                cudaStream_t stream)
 {
-    const unsigned mode = launch_mode(flags, count * 2 * (size_t)nranks);
-    const size_t nvec = count / kVecElems;
+    // chunk = ceil(count / N) rounded up to whole vectors
+    const size_t chunk_vec = ceil_div(ceil_div(count, (size_t)nranks), elems_per_vec(dtype));
+    return dispatch(nranks, u, dtype, [&](auto n_, auto u_, auto d_) -> int {
+        NUNA_NUD(n_, u_, d_);
+        static int occ = 0;
+        auto k = k_twoshot_fused<N, U, DT>;
+        const size_t tiles_per_chunk = ceil_div(chunk_vec, (size_t)kThreads * U);
+        // every block must be resident for the flag barrier: never more than the device holds at once
+        size_t cap = (size_t)num_sms * (size_t)occupancy(nullptr, k, &occ);
+        if (blocks_override > 0) cap = std::min<size_t>(cap, (size_t)blocks_override);
+        const unsigned grid = (unsigned)std::max<size_t>(1, std::min(tiles_per_chunk * N, cap));
+        return launch(k, grid, stream, kLaunchCooperative, p, scratch, count, chunk_vec, bw, timeout_ns);
+    });
+}
+
+int launch_twoshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t count, unsigned flags, cudaStream_t stream)
+{
+    const size_t epv = elems_per_vec(dtype);
+    const unsigned mode = launch_mode(flags, count * elem_size(dtype) * (size_t)nranks);
+    const size_t nvec = count / epv;
     if (flags & NUNA_TWOSHOT_PUT) {
-        return dispatch(nranks, pick_unroll(c, nranks), [&](auto n_, auto u_) -> int {
-            NUNA_NU(n_, u_);
+        return dispatch(nranks, pick_unroll(c, nranks), dtype, [&](auto n_, auto u_, auto d_) -> int {
+            NUNA_NUD(n_, u_, d_);
             static int occ = 0;
-            auto k = k_twoshot_put<N, U>;
+            auto k = k_twoshot_put<N, U, DT>;
             const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
             const unsigned grid = pick_grid(c, std::max<size_t>(ntiles, 1), occupancy(c, k, &occ), 0);
             return launch(k, grid, stream, mode, p, count, ntiles);
         });
     }
-    // chunk = ceil(count / N) rounded up to whole vectors
-    const size_t chunk_vec = ceil_div(ceil_div(count, (size_t)nranks), (size_t)kVecElems);
-    return dispatch(nranks, pick_unroll(c, nranks), [&](auto n_, auto u_) -> int {
-        NUNA_NU(n_, u_);
-        static int occ = 0;
-        auto k = k_twoshot_fused<N, U>;
-        const size_t tiles_per_chunk = ceil_div(chunk_vec, (size_t)kThreads * U);
-        // every block must be resident for the flag barrier: never more than the device holds at once
-        size_t cap = (size_t)c->num_sms * (size_t)occupancy(c, k, &occ);
-        if (c->blocks_override > 0) cap = std::min<size_t>(cap, (size_t)c->blocks_override);
-        const unsigned grid = (unsigned)std::max<size_t>(1, std::min(tiles_per_chunk * N, cap));
-        return launch(k, grid, stream, kLaunchCooperative, p, reinterpret_cast<uint4*>(c->scratch), count, chunk_vec,
-                      c->bw, c->timeout_ns);
-    });
+    return launch_twoshot_fused(c->num_sms, c->blocks_override, p, nranks, dtype, count, pick_unroll(c, nranks),
+                                reinterpret_cast<uint4*>(c->scratch), c->bw, c->timeout_ns, stream);
 }
 
-int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shard, unsigned flags, cudaStream_t stream)
+int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, int dtype, size_t shard, unsigned flags,
+                          cudaStream_t stream)
 {
+    const size_t epv = elems_per_vec(dtype);
     const unsigned mode = launch_mode(flags);
-    if (shard % kVecElems) {
+    if (shard % epv) {
         const unsigned grid = pick_grid(c, ceil_div(shard * nranks, kThreads), 8);
-        return dispatch(nranks, 1, [&](auto n_, auto u_) -> int {
-            NUNA_NU(n_, u_);
-            return launch(k_reduce_scatter_scalar<N>, grid, stream, mode, p, shard);
+        return dispatch(nranks, 1, dtype, [&](auto n_, auto u_, auto d_) -> int {
+            NUNA_NUD(n_, u_, d_);
+            return launch(k_reduce_scatter_scalar<N, DT>, grid, stream, mode, p, shard);
         });
     }
-    const size_t shard_vec = shard / kVecElems;
-    return dispatch(nranks, pick_unroll(c, nranks), [&](auto n_, auto u_) -> int {
-        NUNA_NU(n_, u_);
+    const size_t shard_vec = shard / epv;
+    return dispatch(nranks, pick_unroll(c, nranks), dtype, [&](auto n_, auto u_, auto d_) -> int {
+        NUNA_NUD(n_, u_, d_);
         static int occ = 0;
-        auto k = k_reduce_scatter<N, U>;
+        auto k = k_reduce_scatter<N, U, DT>;
         const size_t tiles = ceil_div(shard_vec, (size_t)kThreads * U);
         const unsigned grid = pick_grid(c, tiles * N, occupancy(c, k, &occ), 0);
         return launch(k, grid, stream, mode, p, shard_vec, tiles);
     });
 }
 
-int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, unsigned flags, cudaStream_t stream)
+// Allgather and alltoall copy bits: they work on 16-byte vectors when a shard is a whole number of
+// them, otherwise on 16-bit units (every element type is a multiple of that).
+int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard_bytes, unsigned flags, cudaStream_t stream)
 {
     const unsigned mode = launch_mode(flags);
-    if (shard % kVecElems) {
-        const unsigned grid = pick_grid(c, ceil_div(shard * nranks, kThreads), 8);
-        return launch(k_allgather_scalar, grid, stream, mode, p, nranks, shard);
+    if (shard_bytes % 16) {
+        const size_t shard16 = shard_bytes / 2;
+        const unsigned grid = pick_grid(c, ceil_div(shard16 * nranks, kThreads), 8);
+        return launch(k_allgather_scalar, grid, stream, mode, p, nranks, shard16);
     }
-    const size_t shard_vec = shard / kVecElems;
+    const size_t shard_vec = shard_bytes / 16;
     static int occ = 0;
     // One block per (rank, tile) storing to all N destinations.  Splitting a tile's destinations over
     // several blocks (dsplit > 1) was measured slower at every size tried (16 x 64 KiB: 4.4 us with 1,
@@ -507,14 +537,15 @@ int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, un
     return launch(k, grid, stream, mode, p, nranks, shard_vec, tiles, dsplit);
 }
 
-int launch_alltoall(Context* c, const RankPtrs& p, int nranks, size_t block, unsigned flags, cudaStream_t stream)
+int launch_alltoall(Context* c, const RankPtrs& p, int nranks, size_t block_bytes, unsigned flags, cudaStream_t stream)
 {
-    const unsigned mode = launch_mode(flags, block * 2 * (size_t)nranks * (size_t)nranks);
-    if (block % kVecElems) {
-        const unsigned grid = pick_grid(c, ceil_div(block * nranks * nranks, kThreads), 8);
-        return launch(k_alltoall_scalar, grid, stream, mode, p, nranks, block);
+    const unsigned mode = launch_mode(flags, block_bytes * (size_t)nranks * (size_t)nranks);
+    if (block_bytes % 16) {
+        const size_t block16 = block_bytes / 2;
+        const unsigned grid = pick_grid(c, ceil_div(block16 * nranks * nranks, kThreads), 8);
+        return launch(k_alltoall_scalar, grid, stream, mode, p, nranks, block16);
     }
-    const size_t block_vec = block / kVecElems;
+    const size_t block_vec = block_bytes / 16;
     static int occ = 0;
     constexpr int U = 2;
     auto k = k_alltoall<U>;
@@ -564,7 +595,7 @@ int nuna_allreduce_oneshot(const void* const* src, void* const* dst, int nranks,
     if (flags & NUNA_TWOSHOT_PUT) return NUNA_ERR_INVALID_ARG;
     Context* c = nullptr;
     if ((st = get_context(&c)) != NUNA_OK) return st;
-    return launch_oneshot(c, make_ptrs(src, dst, nranks), nranks, count, flags, (cudaStream_t)stream);
+    return launch_oneshot(c, make_ptrs(src, dst, nranks), nranks, dtype, count, flags, (cudaStream_t)stream);
 }
 
 int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
@@ -576,7 +607,7 @@ int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
     if ((st = get_context(&c)) != NUNA_OK) return st;
     if (!(flags & NUNA_TWOSHOT_PUT)) {
         std::lock_guard<std::mutex> lock(c->mutex);
-        const size_t need = (count * 2 + 15) & ~(size_t)15;
+        const size_t need = (count * elem_size(dtype) + 15) & ~(size_t)15;
         if (need > c->scratch_bytes) {
             cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
             if (cudaStreamIsCapturing((cudaStream_t)stream, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone)
@@ -584,7 +615,7 @@ int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
             if ((st = ensure_scratch(c, need)) != NUNA_OK) return st;
         }
     }
-    return launch_twoshot(c, make_ptrs(src, dst, nranks), nranks, count, flags, (cudaStream_t)stream);
+    return launch_twoshot(c, make_ptrs(src, dst, nranks), nranks, dtype, count, flags, (cudaStream_t)stream);
 }
 
 int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks, size_t shard_count, int dtype,
@@ -598,7 +629,7 @@ int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks, si
     if (flags & NUNA_TWOSHOT_PUT) return NUNA_ERR_INVALID_ARG;
     Context* c = nullptr;
     if ((st = get_context(&c)) != NUNA_OK) return st;
-    return launch_reduce_scatter(c, make_ptrs(src, dst, nranks), nranks, shard_count, flags, (cudaStream_t)stream);
+    return launch_reduce_scatter(c, make_ptrs(src, dst, nranks), nranks, dtype, shard_count, flags, (cudaStream_t)stream);
 }
 
 int nuna_allgather(const void* const* src, void* const* dst, int nranks, size_t shard_count, int dtype,
@@ -612,7 +643,7 @@ int nuna_allgather(const void* const* src, void* const* dst, int nranks, size_t 
     if (flags & NUNA_TWOSHOT_PUT) return NUNA_ERR_INVALID_ARG;
     Context* c = nullptr;
     if ((st = get_context(&c)) != NUNA_OK) return st;
-    return launch_allgather(c, make_ptrs(src, dst, nranks), nranks, shard_count, flags, (cudaStream_t)stream);
+    return launch_allgather(c, make_ptrs(src, dst, nranks), nranks, shard_count * elem_size(dtype), flags, (cudaStream_t)stream);
 }
 
 int nuna_alltoall(const void* const* src, void* const* dst, int nranks, size_t block_count, int dtype,
@@ -626,7 +657,7 @@ int nuna_alltoall(const void* const* src, void* const* dst, int nranks, size_t b
     if (flags & NUNA_TWOSHOT_PUT) return NUNA_ERR_INVALID_ARG;
     Context* c = nullptr;
     if ((st = get_context(&c)) != NUNA_OK) return st;
-    return launch_alltoall(c, make_ptrs(src, dst, nranks), nranks, block_count, flags, (cudaStream_t)stream);
+    return launch_alltoall(c, make_ptrs(src, dst, nranks), nranks, block_count * elem_size(dtype), flags, (cudaStream_t)stream);
 }
 
 int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
@@ -638,7 +669,7 @@ int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks, si
     Context* c = nullptr;
     if ((st = get_context(&c)) != NUNA_OK) return st;
     std::lock_guard<std::mutex> lock(c->mutex);
-    const size_t bytes = count * 2;
+    const size_t bytes = count * elem_size(dtype);
     const size_t slot = (bytes + 255) & ~(size_t)255;
     const size_t need = slot * 2 * (size_t)nranks;
     if (need > c->staging_bytes) {
@@ -660,8 +691,8 @@ int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks, si
             return NUNA_ERR_CUDA;
     }
     const RankPtrs p = make_ptrs(dsrc, ddst, nranks);
-    st = two_shot ? launch_twoshot(c, p, nranks, count, flags, c->stream)
-                  : launch_oneshot(c, p, nranks, count, flags, c->stream);
+    st = two_shot ? launch_twoshot(c, p, nranks, dtype, count, flags, c->stream)
+                  : launch_oneshot(c, p, nranks, dtype, count, flags, c->stream);
     if (st != NUNA_OK) return st;
     for (int d = 0; d < nranks; ++d)
         if (cudaMemcpyAsync(dst[d], ddst[d], bytes, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
@@ -819,25 +850,15 @@ extern "C" int nuna_allreduce_twoshot_static(const void* const* src, void* const
 {
     int st = check_args(src, dst, nranks, count, count, dtype, 0u, true);
     if (st != NUNA_OK || count == 0) return st;
-    if (count > (size_t)NUNA_STATIC_MAX_COUNT) {
-        fprintf(stderr, "nuna_allreduce_twoshot_static: count %zu exceeds NUNA_STATIC_MAX_COUNT (%d elements); "
-                        "use nuna_allreduce_twoshot for larger messages\n", count, (int)NUNA_STATIC_MAX_COUNT);
+    if (count * elem_size(dtype) > (size_t)NUNA_STATIC_MAX_COUNT * 2) {
+        fprintf(stderr, "nuna_allreduce_twoshot_static: %zu bytes per rank exceed the fixed scratch array "
+                        "(NUNA_STATIC_MAX_COUNT = %d 16-bit elements, %d bytes); use nuna_allreduce_twoshot for larger "
+                        "messages\n", count * elem_size(dtype), (int)NUNA_STATIC_MAX_COUNT, (int)NUNA_STATIC_MAX_COUNT * 2);
         return NUNA_ERR_TOO_LARGE;
     }
     StaticSetup* s = nullptr;
     if ((st = static_setup(&s)) != NUNA_OK) return st;
-    const RankPtrs p = make_ptrs(src, dst, nranks);
-    const size_t chunk_vec = ceil_div(ceil_div(count, (size_t)nranks), (size_t)kVecElems);
     const int u = nranks >= 8 ? 1 : nranks >= 4 ? 2 : 4;
-    return dispatch(nranks, u, [&](auto n_, auto u_) -> int {
-        NUNA_NU(n_, u_);
-        static int occ = 0;
-        auto k = k_twoshot_fused<N, U>;
-        const size_t tiles_per_chunk = ceil_div(chunk_vec, (size_t)kThreads * U);
-        const size_t cap = (size_t)s->num_sms * (size_t)occupancy(nullptr, k, &occ);   // all blocks co-resident
-        const unsigned grid = (unsigned)std::max<size_t>(1, std::min(tiles_per_chunk * N, cap));
-        return launch(k, grid, (cudaStream_t)stream, kLaunchCooperative, p, s->shard, count, chunk_vec, s->barrier,
-                      1000000000ull);
-    });
+    return launch_twoshot_fused(s->num_sms, 0, make_ptrs(src, dst, nranks), nranks, dtype, count, u, s->shard, s->barrier,
+                                1000000000ull, (cudaStream_t)stream);
 }
-

@@ -42,9 +42,9 @@ int nuna_chain_create(const void* const* src_sets, void* const* dst_sets, int ns
     if (st != NUNA_OK) return st;
     if (two_shot && !(flags & NUNA_TWOSHOT_PUT)) {
         std::lock_guard<std::mutex> lock(c->mutex);
-        if ((st = ensure_scratch(c, (count * 2 + 15) & ~(size_t)15)) != NUNA_OK) return st;
+        if ((st = ensure_scratch(c, (count * elem_size(dtype) + 15) & ~(size_t)15)) != NUNA_OK) return st;
     }
-    if (!two_shot && (st = prepare_oneshot(c, nranks, count, flags)) != NUNA_OK) return st;
+    if (!two_shot && (st = prepare_oneshot(c, nranks, dtype, count, flags)) != NUNA_OK) return st;
     cudaStream_t cap = nullptr;
     if (cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking) != cudaSuccess) return NUNA_ERR_CUDA;
     cudaGraph_t graph = nullptr;
@@ -60,7 +60,8 @@ int nuna_chain_create(const void* const* src_sets, void* const* dst_sets, int ns
             p.src[r] = reinterpret_cast<const uint4*>(src_sets[(size_t)s * nranks + r]);
             p.dst[r] = reinterpret_cast<uint4*>(dst_sets[(size_t)s * nranks + r]);
         }
-        st = two_shot ? launch_twoshot(c, p, nranks, count, flags, cap) : launch_oneshot(c, p, nranks, count, flags, cap);
+        st = two_shot ? launch_twoshot(c, p, nranks, dtype, count, flags, cap)
+                      : launch_oneshot(c, p, nranks, dtype, count, flags, cap);
     }
     const cudaError_t e = cudaStreamEndCapture(cap, &graph);
     cudaStreamDestroy(cap);

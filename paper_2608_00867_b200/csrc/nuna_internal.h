@@ -56,10 +56,12 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
                int dtype, unsigned flags, bool device_ptrs);
 void plan_oneshot_lists(const nuna_topology_t* topo, int num_sms, int nranks, size_t ntiles, size_t tile_bytes,
                         bool generic, std::vector<std::vector<unsigned>>& lists);
-int prepare_oneshot(Context* c, int nranks, size_t count, unsigned flags);
-int launch_oneshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream);
-int launch_twoshot(Context* c, const RankPtrs& p, int nranks, size_t count, unsigned flags, cudaStream_t stream);
-int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, size_t shard, unsigned flags, cudaStream_t stream);
-int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard, unsigned flags, cudaStream_t stream);
+size_t elem_size(int dtype);
+int prepare_oneshot(Context* c, int nranks, int dtype, size_t count, unsigned flags);
+int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t count, unsigned flags, cudaStream_t stream);
+int launch_twoshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t count, unsigned flags, cudaStream_t stream);
+int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, int dtype, size_t shard, unsigned flags,
+                          cudaStream_t stream);
+int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard_bytes, unsigned flags, cudaStream_t stream);
 
 }  // namespace nuna

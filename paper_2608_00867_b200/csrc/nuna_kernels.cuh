@@ -83,63 +83,132 @@ __device__ __forceinline__ uint16_t ld_src16(const uint16_t* p)
 
 // ---- the fold ------------------------------------------------------------------------------
 
-// bf16 -> binary32 is a 16-bit shift; a 32-bit word holds element 2k in its low half and 2k+1
-// in its high half.  Rank 0's value is widened with a shift / mask; ranks 1..N-1 are folded in with
-// the sm_100 mixed-precision add, d = f32(bf16 a) + c rounded once to binary32 (nearest even,
-// subnormals kept), so no instruction is spent on widening them.  At large sizes the one-shot is
-// limited by instruction issue and L1 throughput (N times the work of a plain sum), which is why
-// the instruction count matters.
-__device__ __forceinline__ float add_bf16(float acc, uint16_t h)
+// Element types (the values of nuna_dtype_t): 0 = bf16, 1 = f16 (IEEE binary16), 2 = f32.
+// Storage is 2 or 4 bytes; a 16-byte vector holds kElems elements; every type is widened exactly
+// to binary32, folded in binary32 in rank order, and rounded once to the storage type.
+constexpr int kBf16 = 0, kF16 = 1, kF32 = 2;
+
+template <int DT> struct Elem { static constexpr int kElems = 8; static constexpr int kBytes = 2; };
+template <> struct Elem<kF32> { static constexpr int kElems = 4; static constexpr int kBytes = 4; };
+
+// bf16 -> binary32 is a 16-bit shift; a 32-bit word holds element 2k in its low half and 2k+1 in
+// its high half.  Rank 0's value is widened (shift / mask for bf16, cvt for f16); ranks 1..N-1 are
+// folded in with the sm_100 mixed-precision add, d = f32(a) + c rounded once to binary32 (nearest
+// even, subnormals kept), so no instruction is spent on widening them.  At large sizes the one-shot is
+// limited by instruction issue and L1 throughput (N times the work of a plain sum), which is why the
+// instruction count matters.
+template <int DT>
+__device__ __forceinline__ float add_narrow(float acc, uint16_t h)
 {
     float d;
-    asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(acc));
+    if (DT == kBf16) asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(acc));
+    else             asm("add.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(acc));
     return d;
 }
 
+template <int DT>
+__device__ __forceinline__ void widen_word(float& lo, float& hi, uint32_t w)
+{
+    if (DT == kBf16) {
+        lo = __uint_as_float(w << 16);
+        hi = __uint_as_float(w & 0xFFFF0000u);
+    } else {
+        uint16_t l, h;
+        asm("mov.b32 {%0, %1}, %2;" : "=h"(l), "=h"(h) : "r"(w));
+        asm("cvt.f32.f16 %0, %1;" : "=f"(lo) : "h"(l));
+        asm("cvt.f32.f16 %0, %1;" : "=f"(hi) : "h"(h));
+    }
+}
+
+template <int DT>
 __device__ __forceinline__ void fold_word(float& lo, float& hi, uint32_t w)
 {
     uint16_t l, h;
     asm("mov.b32 {%0, %1}, %2;" : "=h"(l), "=h"(h) : "r"(w));
-    lo = add_bf16(lo, l);
-    hi = add_bf16(hi, h);
+    lo = add_narrow<DT>(lo, l);
+    hi = add_narrow<DT>(hi, h);
 }
 
-// Two binary32 -> one word of two bf16, round to nearest even, NaN -> 0x7FFF.
+// Two binary32 -> one word of two 16-bit elements, round to nearest even, NaN -> 0x7FFF.
+template <int DT>
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     uint32_t d;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    if (DT == kBf16) asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    else             asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
 }
 
 // Fold N already-loaded vectors in rank order: acc starts from rank 0's value, N-1 additions.
-template <int N>
+template <int N, int DT>
 __device__ __forceinline__ uint4 fold_vectors(const uint4 (&v)[N])
 {
+    if (DT == kF32) {
+        float a0 = __uint_as_float(v[0].x), a1 = __uint_as_float(v[0].y);
+        float a2 = __uint_as_float(v[0].z), a3 = __uint_as_float(v[0].w);
+#pragma unroll
+        for (int r = 1; r < N; ++r) {
+            a0 = __fadd_rn(a0, __uint_as_float(v[r].x));
+            a1 = __fadd_rn(a1, __uint_as_float(v[r].y));
+            a2 = __fadd_rn(a2, __uint_as_float(v[r].z));
+            a3 = __fadd_rn(a3, __uint_as_float(v[r].w));
+        }
+        return make_uint4(__float_as_uint(a0), __float_as_uint(a1), __float_as_uint(a2), __float_as_uint(a3));
+    }
     float a[8];
-    a[0] = __uint_as_float(v[0].x << 16); a[1] = __uint_as_float(v[0].x & 0xFFFF0000u);
-    a[2] = __uint_as_float(v[0].y << 16); a[3] = __uint_as_float(v[0].y & 0xFFFF0000u);
-    a[4] = __uint_as_float(v[0].z << 16); a[5] = __uint_as_float(v[0].z & 0xFFFF0000u);
-    a[6] = __uint_as_float(v[0].w << 16); a[7] = __uint_as_float(v[0].w & 0xFFFF0000u);
+    widen_word<DT>(a[0], a[1], v[0].x);
+    widen_word<DT>(a[2], a[3], v[0].y);
+    widen_word<DT>(a[4], a[5], v[0].z);
+    widen_word<DT>(a[6], a[7], v[0].w);
 #pragma unroll
     for (int r = 1; r < N; ++r) {
-        fold_word(a[0], a[1], v[r].x);
-        fold_word(a[2], a[3], v[r].y);
-        fold_word(a[4], a[5], v[r].z);
-        fold_word(a[6], a[7], v[r].w);
+        fold_word<DT>(a[0], a[1], v[r].x);
+        fold_word<DT>(a[2], a[3], v[r].y);
+        fold_word<DT>(a[4], a[5], v[r].z);
+        fold_word<DT>(a[6], a[7], v[r].w);
     }
-    return make_uint4(pack2(a[0], a[1]), pack2(a[2], a[3]), pack2(a[4], a[5]), pack2(a[6], a[7]));
+    return make_uint4(pack2<DT>(a[0], a[1]), pack2<DT>(a[2], a[3]), pack2<DT>(a[4], a[5]), pack2<DT>(a[6], a[7]));
 }
 
-// One element (ragged tails and unaligned shards).
-template <int N>
-__device__ __forceinline__ uint16_t fold_scalar(const RankPtrs& p, size_t elem)
+// One element (ragged tails and unaligned shards): returns the storage word of the folded value.
+template <int N, int DT>
+__device__ __forceinline__ uint32_t fold_scalar(const RankPtrs& p, size_t elem)
 {
-    float acc = __uint_as_float((uint32_t)ld_src16(reinterpret_cast<const uint16_t*>(p.src[0]) + elem) << 16);
+    if (DT == kF32) {
+        float acc = __uint_as_float(__ldg(reinterpret_cast<const uint32_t*>(p.src[0]) + elem));
+#pragma unroll
+        for (int r = 1; r < N; ++r)
+            acc = __fadd_rn(acc, __uint_as_float(__ldg(reinterpret_cast<const uint32_t*>(p.src[r]) + elem)));
+        return __float_as_uint(acc);
+    }
+    float acc, unused;
+    widen_word<DT>(acc, unused, (uint32_t)ld_src16(reinterpret_cast<const uint16_t*>(p.src[0]) + elem));
 #pragma unroll
     for (int r = 1; r < N; ++r)
-        acc = __fadd_rn(acc, __uint_as_float((uint32_t)ld_src16(reinterpret_cast<const uint16_t*>(p.src[r]) + elem) << 16));
-    return (uint16_t)(pack2(acc, 0.0f) & 0xFFFFu);
+        acc = add_narrow<DT>(acc, ld_src16(reinterpret_cast<const uint16_t*>(p.src[r]) + elem));
+    return pack2<DT>(acc, 0.0f) & 0xFFFFu;
+}
+
+template <int DT>
+__device__ __forceinline__ void store_elem(void* base, size_t elem, uint32_t word)
+{
+    if (DT == kF32) reinterpret_cast<uint32_t*>(base)[elem] = word;
+    else            reinterpret_cast<uint16_t*>(base)[elem] = (uint16_t)word;
+}
+
+// Element written earlier in this kernel by another block: L2-coherent load.
+template <int DT>
+__device__ __forceinline__ uint32_t load_elem_cg(const void* base, size_t elem)
+{
+    uint32_t w;
+    if (DT == kF32) {
+        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(w) : "l"(reinterpret_cast<const uint32_t*>(base) + elem) : "memory");
+    } else {
+        uint16_t v;
+        asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(v) : "l"(reinterpret_cast<const uint16_t*>(base) + elem) : "memory");
+        w = v;
+    }
+    return w;
 }
 
 // ---- one-shot allreduce: work item = (tile, destination rank) ---------------------------------
@@ -148,7 +217,7 @@ __device__ __forceinline__ uint16_t fold_scalar(const RankPtrs& p, size_t elem)
 // the same source tile are adjacent in the item order.  A tile is
 // kThreads * U vectors.  Round-robin placement: item i is taken by block
 // i mod gridDim.x (the locality-unaware baseline of Section 5.3).
-template <int N, int U>
+template <int N, int U, int DT>
 __device__ __forceinline__ void oneshot_item(const RankPtrs& p, size_t nvec, size_t tile, int d)
 {
     const size_t base = tile * (size_t)(kThreads * U) + threadIdx.x;
@@ -164,26 +233,26 @@ __device__ __forceinline__ void oneshot_item(const RankPtrs& p, size_t nvec, siz
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const size_t i = base + (size_t)u * kThreads;
-        if (i < nvec) st_dst(p.dst[d] + i, fold_vectors<N>(v[u]));
+        if (i < nvec) st_dst(p.dst[d] + i, fold_vectors<N, DT>(v[u]));
     }
 }
 
-template <int N, int U>
+template <int N, int U, int DT>
 __global__ void __launch_bounds__(kThreads, min_blocks(N * U))
 k_oneshot_rr(const RankPtrs p, const size_t count, const size_t ntiles)
 {
     pdl_wait();
-    const size_t nvec = count / kVecElems;
+    const size_t nvec = count / Elem<DT>::kElems;
     const size_t nitems = ntiles * N;
     for (size_t item = blockIdx.x; item < nitems; item += gridDim.x)
-        oneshot_item<N, U>(p, nvec, item / N, (int)(item % N));
+        oneshot_item<N, U, DT>(p, nvec, item / N, (int)(item % N));
     pdl_trigger();
     // ragged tail (count % 8 elements): block d handles destination d
-    const size_t tail0 = nvec * kVecElems;
+    const size_t tail0 = nvec * Elem<DT>::kElems;
     if (tail0 < count) {
         for (int d = blockIdx.x; d < N; d += gridDim.x) {
             const size_t e = tail0 + threadIdx.x;
-            if (e < count) reinterpret_cast<uint16_t*>(p.dst[d])[e] = fold_scalar<N>(p, e);
+            if (e < count) store_elem<DT>(p.dst[d], e, fold_scalar<N, DT>(p, e));
         }
     }
 }
@@ -211,7 +280,7 @@ __device__ __forceinline__ uint4 ld_src_l1(const uint4* p)
 // resource budget of Section 4.2.2 in SM terms: the more items of a group share an SM, the fewer
 // distinct bytes that SM has in flight (kThreads / C vectors per source), so cold data wants a small
 // C (more outstanding requests per SM) and L2-resident data a large one (fewer L2 -> SM transfers).
-template <int N, int C>
+template <int N, int C, int DT>
 __device__ __forceinline__ void oneshot_group(const RankPtrs& p, size_t nvec, size_t tile, int dst0)
 {
     constexpr int kLanes = kThreads / C;                 // vectors per tile
@@ -221,26 +290,26 @@ __device__ __forceinline__ void oneshot_group(const RankPtrs& p, size_t nvec, si
         uint4 v[N];
 #pragma unroll
         for (int r = 0; r < N; ++r) v[r] = ld_src_l1(p.src[r] + i);
-        st_dst(p.dst[d] + i, fold_vectors<N>(v));
+        st_dst(p.dst[d] + i, fold_vectors<N, DT>(v));
     }
 }
 
-template <int N, int C>
+template <int N, int C, int DT>
 __global__ void __launch_bounds__(kThreads, min_blocks(N))
 k_oneshot_group(const RankPtrs p, const size_t count, const size_t ntiles)
 {
     pdl_wait();
     constexpr int kSplit = (N + C - 1) / C;              // blocks per tile group
-    const size_t nvec = count / kVecElems;
+    const size_t nvec = count / Elem<DT>::kElems;
     const size_t nitems = ntiles * kSplit;
     for (size_t it = blockIdx.x; it < nitems; it += gridDim.x)
-        oneshot_group<N, C>(p, nvec, it / kSplit, (int)(it % kSplit) * C);
+        oneshot_group<N, C, DT>(p, nvec, it / kSplit, (int)(it % kSplit) * C);
     pdl_trigger();
-    const size_t tail0 = nvec * kVecElems;
+    const size_t tail0 = nvec * Elem<DT>::kElems;
     if (tail0 < count) {
         for (int d = blockIdx.x; d < N; d += gridDim.x) {
             const size_t e = tail0 + threadIdx.x;
-            if (e < count) reinterpret_cast<uint16_t*>(p.dst[d])[e] = fold_scalar<N>(p, e);
+            if (e < count) store_elem<DT>(p.dst[d], e, fold_scalar<N, DT>(p, e));
         }
     }
 }
@@ -316,7 +385,7 @@ __device__ __forceinline__ unsigned find_orphan(const SmLists& sl, unsigned own)
     return 0xFFFFFFFFu;
 }
 
-template <int N, int C>
+template <int N, int C, int DT>
 __global__ void __launch_bounds__(kThreads, min_blocks(N))
 k_oneshot_sm(const RankPtrs p, const size_t count, const SmLists sl, const unsigned blocks_per_sm)
 {
@@ -324,7 +393,7 @@ k_oneshot_sm(const RankPtrs p, const size_t count, const SmLists sl, const unsig
     constexpr int kSplit = (N + C - 1) / C;
     __shared__ unsigned sh_n;
     __shared__ unsigned sh_tiles[kMaxBatch];
-    const size_t nvec = count / kVecElems;
+    const size_t nvec = count / Elem<DT>::kElems;
     const unsigned own = read_smid_reg() % (unsigned)sl.num_sms;
     const unsigned own_len = sl.off[own + 1] - sl.off[own];
     // an SM's list is shared by the blocks resident there: one claim per block takes its whole share
@@ -363,17 +432,17 @@ k_oneshot_sm(const RankPtrs p, const size_t count, const SmLists sl, const unsig
             for (unsigned i = 0; i < n; ++i) {
                 const size_t tile = sh_tiles[i];
 #pragma unroll
-                for (int sub = 0; sub < kSplit; ++sub) oneshot_group<N, C>(p, nvec, tile, sub * C);
+                for (int sub = 0; sub < kSplit; ++sub) oneshot_group<N, C, DT>(p, nvec, tile, sub * C);
             }
         }
         __syncthreads();
     }
     pdl_trigger();
-    const size_t tail0 = nvec * kVecElems;
+    const size_t tail0 = nvec * Elem<DT>::kElems;
     if (tail0 < count) {
         for (int d = blockIdx.x; d < N; d += gridDim.x) {
             const size_t e = tail0 + threadIdx.x;
-            if (e < count) reinterpret_cast<uint16_t*>(p.dst[d])[e] = fold_scalar<N>(p, e);
+            if (e < count) store_elem<DT>(p.dst[d], e, fold_scalar<N, DT>(p, e));
         }
     }
     // the last block out rewinds cursors, presence flags and counters for the next launch
@@ -392,7 +461,7 @@ k_oneshot_sm(const RankPtrs p, const size_t count, const SmLists sl, const unsig
 //
 // dst[r][j] = fold_k src[k][r*S + j].  `shard_vec` = S/8 (vector path requires S % 8 == 0, which
 // keeps r*S 16-byte aligned); `out` overrides dst (the fused two-shot writes into its shard scratch).
-template <int N, int U>
+template <int N, int U, int DT>
 __device__ __forceinline__ void reduce_tile(const RankPtrs& p, uint4* out, size_t src_off_vec,
                                             size_t nvec, size_t tile)
 {
@@ -409,11 +478,11 @@ __device__ __forceinline__ void reduce_tile(const RankPtrs& p, uint4* out, size_
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const size_t i = base + (size_t)u * kThreads;
-        if (i < nvec) st_dst(out + i, fold_vectors<N>(v[u]));
+        if (i < nvec) st_dst(out + i, fold_vectors<N, DT>(v[u]));
     }
 }
 
-template <int N, int U>
+template <int N, int U, int DT>
 __global__ void __launch_bounds__(kThreads, min_blocks(N * U))
 k_reduce_scatter(const RankPtrs p, const size_t shard_vec, const size_t tiles_per_shard)
 {
@@ -422,13 +491,13 @@ k_reduce_scatter(const RankPtrs p, const size_t shard_vec, const size_t tiles_pe
     for (size_t item = blockIdx.x; item < nitems; item += gridDim.x) {
         const int r = (int)(item / tiles_per_shard);
         const size_t tile = item % tiles_per_shard;
-        reduce_tile<N, U>(p, p.dst[r], (size_t)r * shard_vec, shard_vec, tile);
+        reduce_tile<N, U, DT>(p, p.dst[r], (size_t)r * shard_vec, shard_vec, tile);
     }
     pdl_trigger();
 }
 
 // Any shard length: one element per thread (slow path, used when S % 8 != 0).
-template <int N>
+template <int N, int DT>
 __global__ void __launch_bounds__(kThreads)
 k_reduce_scatter_scalar(const RankPtrs p, const size_t shard)
 {
@@ -436,7 +505,7 @@ k_reduce_scatter_scalar(const RankPtrs p, const size_t shard)
     const size_t total = shard * N;
     for (size_t e = (size_t)blockIdx.x * kThreads + threadIdx.x; e < total; e += (size_t)gridDim.x * kThreads) {
         const int r = (int)(e / shard);
-        reinterpret_cast<uint16_t*>(p.dst[r])[e - (size_t)r * shard] = fold_scalar<N>(p, e);
+        store_elem<DT>(p.dst[r], e - (size_t)r * shard, fold_scalar<N, DT>(p, e));
     }
 }
 
@@ -608,12 +677,12 @@ __device__ __forceinline__ bool flag_barrier(BarrierWords* bw, unsigned int expe
 // whose outputs live side by side in `scratch`).  Flag barrier.  Phase 2: put-style
 // allgather, chunk r is loaded once and stored into all N destinations.
 // chunk_vec = vectors per chunk; the last chunks may be short or empty.
-template <int N, int U>
+template <int N, int U, int DT>
 __global__ void __launch_bounds__(kThreads, min_blocks(N * U))
 k_twoshot_fused(const RankPtrs p, uint4* scratch, const size_t count, const size_t chunk_vec,
                 BarrierWords* bw, const unsigned long long timeout_ns)
 {
-    const size_t nvec = count / kVecElems;
+    const size_t nvec = count / Elem<DT>::kElems;
     const size_t tiles_per_chunk = (chunk_vec + kThreads * U - 1) / (kThreads * U);
     const size_t nitems = tiles_per_chunk * N;
     __shared__ unsigned sh_item;
@@ -643,12 +712,12 @@ k_twoshot_fused(const RankPtrs p, uint4* scratch, const size_t count, const size
         const size_t off = (size_t)r * chunk_vec;
         if (off >= nvec) return;
         const size_t len = (nvec - off < chunk_vec) ? nvec - off : chunk_vec;
-        reduce_tile<N, U>(p, scratch + off, off, len, tile);
+        reduce_tile<N, U, DT>(p, scratch + off, off, len, tile);
     });
-    const size_t tail0 = nvec * kVecElems;             // ragged tail: reduced by block 0 into scratch
+    const size_t tail0 = nvec * Elem<DT>::kElems;             // ragged tail: reduced by block 0 into scratch
     if (tail0 < count && blockIdx.x == 0) {
         const size_t e = tail0 + threadIdx.x;
-        if (e < count) reinterpret_cast<uint16_t*>(scratch)[e] = fold_scalar<N>(p, e);
+        if (e < count) store_elem<DT>(scratch, e, fold_scalar<N, DT>(p, e));
     }
 
     if (!flag_barrier(bw, gridDim.x, epoch0, timeout_ns)) return;
@@ -664,20 +733,19 @@ k_twoshot_fused(const RankPtrs p, uint4* scratch, const size_t count, const size
     if (tail0 < count && blockIdx.x == 0) {
         const size_t e = tail0 + threadIdx.x;
         if (e < count) {
-            uint16_t v;
-            asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(v) : "l"(reinterpret_cast<uint16_t*>(scratch) + e) : "memory");
-            for (int d = 0; d < N; ++d) reinterpret_cast<uint16_t*>(p.dst[d])[e] = v;
+            const uint32_t v = load_elem_cg<DT>(scratch, e);
+            for (int d = 0; d < N; ++d) store_elem<DT>(p.dst[d], e, v);
         }
     }
 }
 
 // Two-shot without the intermediate: the block that reduces a tile stores it into all N destinations.
-template <int N, int U>
+template <int N, int U, int DT>
 __global__ void __launch_bounds__(kThreads, min_blocks(N * U))
 k_twoshot_put(const RankPtrs p, const size_t count, const size_t ntiles)
 {
     pdl_wait();
-    const size_t nvec = count / kVecElems;
+    const size_t nvec = count / Elem<DT>::kElems;
     for (size_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const size_t base = tile * (size_t)(kThreads * U) + threadIdx.x;
         uint4 v[U][N];
@@ -693,19 +761,19 @@ k_twoshot_put(const RankPtrs p, const size_t count, const size_t ntiles)
         for (int u = 0; u < U; ++u) {
             const size_t i = base + (size_t)u * kThreads;
             if (i < nvec) {
-                const uint4 o = fold_vectors<N>(v[u]);
+                const uint4 o = fold_vectors<N, DT>(v[u]);
 #pragma unroll
                 for (int d = 0; d < N; ++d) st_dst(p.dst[d] + i, o);
             }
         }
     }
     pdl_trigger();
-    const size_t tail0 = nvec * kVecElems;
+    const size_t tail0 = nvec * Elem<DT>::kElems;
     if (tail0 < count && blockIdx.x == 0) {
         const size_t e = tail0 + threadIdx.x;
         if (e < count) {
-            const uint16_t v = fold_scalar<N>(p, e);
-            for (int d = 0; d < N; ++d) reinterpret_cast<uint16_t*>(p.dst[d])[e] = v;
+            const uint32_t v = fold_scalar<N, DT>(p, e);
+            for (int d = 0; d < N; ++d) store_elem<DT>(p.dst[d], e, v);
         }
     }
 }

@@ -7,7 +7,6 @@ namespace nuna {
 
 constexpr int kMaxRanks = 16;
 constexpr int kThreads = 256;            // threads per block, every kernel
-constexpr int kVecElems = 8;             // bf16 per 16-byte vector
 
 // Kernel argument: the rank buffers, by value.
 struct RankPtrs {

@@ -50,7 +50,9 @@ def test_validation_happens_before_any_cuda_call():
     assert call([], [], 0, nranks=0) == nb.NUNA_ERR_INVALID_ARG
     assert call(ok_src, ok_dst, 0) == nb.NUNA_OK                               # empty: no launch, no context
     assert call(ok_src * 9, ok_dst * 9, 8) == nb.NUNA_ERR_TOO_MANY_RANKS
-    assert call(ok_src, ok_dst, 8, dtype=nb.NUNA_F16) == nb.NUNA_ERR_UNSUPPORTED_DTYPE
+    assert call(ok_src, ok_dst, 8, dtype=nb.NUNA_F16) in (nb.NUNA_ERR_CUDA, nb.NUNA_OK)   # valid type; no device here
+    assert call(ok_src, [A + 8192, A + 8192 + 16], 5, dtype=nb.NUNA_F32) == nb.NUNA_ERR_ALIAS   # 20 bytes each: overlap
+    assert call(ok_src, [A + 8192, A + 8192 + 16], 5, dtype=nb.NUNA_BF16) in (nb.NUNA_ERR_CUDA, nb.NUNA_OK)  # 10 bytes: fine
     assert call(ok_src, ok_dst, 8, dtype=77) == nb.NUNA_ERR_UNSUPPORTED_DTYPE
     assert call(ok_src, ok_dst, 8, flags=3) == nb.NUNA_ERR_INVALID_ARG
     assert call(ok_src, ok_dst, 8, flags=1 << 9) == nb.NUNA_ERR_INVALID_ARG

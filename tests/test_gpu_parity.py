@@ -378,7 +378,7 @@ def test_argument_errors_launch_nothing():
     assert nb.nuna_allreduce_oneshot(a, [b[0], b[0]], 64, check=False) == nb.NUNA_ERR_ALIAS
     assert nb.nuna_allreduce_oneshot(a, [b[0], a[1][16:]], 32, check=False) == nb.NUNA_ERR_ALIAS
     assert nb.nuna_allreduce_oneshot(a, [b[0], b[1][1:]], 8, check=False) == nb.NUNA_ERR_ALIGNMENT
-    assert nb.nuna_allreduce_oneshot(a, b, 64, dtype=nb.NUNA_F32, check=False) == nb.NUNA_ERR_UNSUPPORTED_DTYPE
+    assert nb.nuna_allreduce_oneshot(a, b, 64, dtype=5, check=False) == nb.NUNA_ERR_UNSUPPORTED_DTYPE
     assert nb.nuna_allreduce_oneshot(a, b, 64, flags=3, check=False) == nb.NUNA_ERR_INVALID_ARG
     assert nb.nuna_allreduce_oneshot(a, b, 64, flags=nb.NUNA_TWOSHOT_PUT, check=False) == nb.NUNA_ERR_INVALID_ARG
     assert nb.nuna_allreduce_oneshot(a * 9, b * 9, 64, check=False) == nb.NUNA_ERR_TOO_MANY_RANKS
