@@ -364,7 +364,7 @@ def run_gpu(args):
             "oneshot_aware": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=nb.NUNA_PLACE_AWARE, stream=st)),
             "twoshot": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, stream=st)),
             "twoshot_put": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, flags=nb.NUNA_TWOSHOT_PUT, stream=st)),
-            # the same two with programmatic dependent launch (dropped by the library above 16 MiB of sources)
+            # the same two with programmatic dependent launch (the one-shot drops it above 16 MiB of sources)
             "oneshot_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=nb.NUNA_LAUNCH_PDL, stream=st)),
             "twoshot_put_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(
                 s, d, c, flags=nb.NUNA_TWOSHOT_PUT | nb.NUNA_LAUNCH_PDL, stream=st)),

@@ -80,7 +80,8 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 /* `flags`, bit 6: launch with programmatic stream serialization.  The kernel may be scheduled while its
  * predecessor in the stream drains; it waits for that grid's completion and memory visibility before
  * its first global access, so results are those of an ordinary stream-ordered launch.  Ignored by the
- * flag-barrier two-shot (a cooperative launch) and above 16 MiB of sources, where it does not pay.     */
+ * flag-barrier two-shot (a cooperative launch) and by the one-shot above 16 MiB of sources, where it
+ * was measured not to pay.                                                                              */
 #define NUNA_LAUNCH_PDL       64u
 /* `flags`, bit 7, with NUNA_PLACE_AWARE on nuna_allreduce_oneshot: dispatch the co-located groups through
  * per-SM work lists.  The lists are planned by Algorithm 1 from the topology the last

@@ -154,7 +154,9 @@ static unsigned pick_grid(const Context* c, size_t nitems, int blocks_per_sm, in
 constexpr unsigned kLaunchPlain = 0u, kLaunchCooperative = 1u, kLaunchPdl = 2u;
 
 // Programmatic dependent launch pays off while a kernel is short enough for its launch latency to
-// matter; from about 16 MiB of sources it was measured to cost a few percent, so it is dropped there.
+// matter.  For the one-shot it was measured to cost a few percent from about 16 MiB of sources (its
+// multi-wave grid competes with the successor's early blocks), so it is dropped there; the streaming
+// kernels (two-shot put, reduce-scatter, allgather) keep it at every size (4 MiB per rank: 12.6 -> 12.0 us).
 static unsigned launch_mode(unsigned flags, size_t total_src_bytes = 0)
 {
     return ((flags & NUNA_LAUNCH_PDL) && total_src_bytes <= ((size_t)16 << 20)) ? kLaunchPdl : kLaunchPlain;
@@ -475,7 +477,7 @@ static int launch_twoshot_fused(int num_sms, int blocks_override, const RankPtrs
 int launch_twoshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t count, unsigned flags, cudaStream_t stream)
 {
     const size_t epv = elems_per_vec(dtype);
-    const unsigned mode = launch_mode(flags, count * elem_size(dtype) * (size_t)nranks);
+    const unsigned mode = launch_mode(flags);
     const size_t nvec = count / epv;
     if (flags & NUNA_TWOSHOT_PUT) {
         return dispatch(nranks, pick_unroll(c, nranks), dtype, [&](auto n_, auto u_, auto d_) -> int {
@@ -539,7 +541,7 @@ int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard_byt
 
 int launch_alltoall(Context* c, const RankPtrs& p, int nranks, size_t block_bytes, unsigned flags, cudaStream_t stream)
 {
-    const unsigned mode = launch_mode(flags, block_bytes * (size_t)nranks * (size_t)nranks);
+    const unsigned mode = launch_mode(flags);
     if (block_bytes % 16) {
         const size_t block16 = block_bytes / 2;
         const unsigned grid = pick_grid(c, ceil_div(block16 * nranks * nranks, kThreads), 8);

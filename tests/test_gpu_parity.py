@@ -359,6 +359,43 @@ def test_tuning_options_change_the_launch_not_the_bits():
     assert nb.nuna_device_status() == nb.NUNA_OK
 
 
+def test_two_host_threads_on_their_own_streams():
+    """Calls that share no library state (one-shot, two-shot put, allgather) may be issued from
+    different host threads on different streams at the same time."""
+    import threading
+    n, count, rounds = 8, 64 * 1024 + 3, 40
+    errors = []
+
+    def worker(tid):
+        try:
+            torch.cuda.set_device(0)
+            stream = torch.cuda.Stream()
+            src = workloads.special_values(n, count, seed=900 + tid)
+            want = oracle.allreduce(src, nthreads=2)[0]
+            with torch.cuda.stream(stream):
+                dsrc = upload(src)
+                dst = [torch.zeros(count, dtype=torch.int16, device="cuda") for _ in range(n)]
+                stream.synchronize()
+                for i in range(rounds):
+                    flags = (0, nb.NUNA_PLACE_AWARE, nb.NUNA_LAUNCH_PDL)[i % 3]
+                    if i % 2:
+                        nb.nuna_allreduce_oneshot(dsrc, dst, count, flags=flags, stream=stream)
+                    else:
+                        nb.nuna_allreduce_twoshot(dsrc, dst, count, flags=nb.NUNA_TWOSHOT_PUT, stream=stream)
+                stream.synchronize()
+                for t in dst:
+                    assert_same_bits(t.cpu().numpy().view(np.uint16), want, f"thread {tid}")
+        except Exception as e:                                     # noqa: BLE001 - reported by the main thread
+            errors.append((tid, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(t,)) for t in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+
+
 def test_host_buffer_entry_point():
     for n, count, two in ((8, 32 * 8192, False), (8, 32 * 8192, True), (3, 1001, False), (3, 1001, True)):
         src = workloads.rank_buffers(n, count, "normal", seed=77)
