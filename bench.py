@@ -356,7 +356,7 @@ def run_gpu(args):
         extras["e2e"] = {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": N_RANKS * w.bytes_per_rank,
                          "d2h_bytes_per_step": N_RANKS * w.bytes_per_rank}
 
-    sweep, ag_row, a2a_row, chain_rows = [], None, None, []
+    sweep, ag_row, a2a_row, rs_rows, chain_rows = [], None, None, [], []
     if not args.quick:
         # ---- message-size sweep, 8 ranks, 8 KiB .. 64 MiB per rank --------------------------------------
         algos = {
@@ -394,18 +394,32 @@ def run_gpu(args):
         # ---- allgather, 16 ranks x 64 KiB ---------------------------------------------------------------
         wa = workloads.config_allgather16()
         asets = make_sets(wa.nranks, wa.count, wa.nranks * wa.count, 2 * l2 + (64 << 20), "uniform", wa.seed)
-        ag_us = per_call_us(lambda s, d, st: nb.nuna_allgather(s, d, wa.count, stream=st), asets, 512, 3)
+        ag_us = per_call_us(lambda s, d, st: nb.nuna_allgather(s, d, wa.count, flags=nb.NUNA_LAUNCH_PDL, stream=st), asets, 512, 3)
         ag_bytes = wa.nranks * wa.bytes_per_rank + wa.nranks * wa.nranks * wa.bytes_per_rank
         ag_row = {"workload": wa.name, "us": round(ag_us, 3), "algorithmic_bytes": ag_bytes,
                   "gbs": round(ag_bytes / ag_us / 1e3, 1), "frac_of_peak": round(ag_bytes / ag_us / 1e3 / peak_gbs, 4)}
         del asets
         torch.cuda.empty_cache()
 
+        # ---- reduce-scatter, 8 ranks, 4 MiB and 32 MiB of sources per rank --------------------------------
+        rs_rows = []
+        for log2b in (22, 25):
+            cnt = (1 << log2b) // 2
+            shard = cnt // N_RANKS
+            rsets = make_sets(N_RANKS, cnt, shard, 2 * l2 + (64 << 20), "normal", 60 + log2b)
+            rs_us = per_call_us(lambda s, d, st: nb.nuna_reduce_scatter(s, d, shard, flags=nb.NUNA_LAUNCH_PDL, stream=st),
+                                rsets, max(len(rsets), 64), 3)
+            rs_bytes = N_RANKS * 2 * cnt + 2 * cnt                     # every source once + every shard once
+            rs_rows.append({"bytes_per_rank": 2 * cnt, "us": round(rs_us, 3), "algorithmic_bytes": rs_bytes,
+                            "gbs": round(rs_bytes / rs_us / 1e3, 1), "frac_of_peak": round(rs_bytes / rs_us / 1e3 / peak_gbs, 4)})
+            del rsets
+            torch.cuda.empty_cache()
+
         # ---- alltoall, 8 ranks x 64 KiB per pair ----------------------------------------------------------
         wt = workloads.config_alltoall8()
         tsets = make_sets(wt.nranks, wt.count, wt.count, 2 * l2 + (64 << 20), "normal", wt.seed)
         blk = wt.count // wt.nranks
-        a2a_us = per_call_us(lambda s, d, st: nb.nuna_alltoall(s, d, blk, stream=st), tsets, 512, 3)
+        a2a_us = per_call_us(lambda s, d, st: nb.nuna_alltoall(s, d, blk, flags=nb.NUNA_LAUNCH_PDL, stream=st), tsets, 512, 3)
         a2a_bytes = 2 * wt.nranks * wt.bytes_per_rank
         a2a_row = {"workload": wt.name, "us": round(a2a_us, 3), "algorithmic_bytes": a2a_bytes,
                    "gbs": round(a2a_bytes / a2a_us / 1e3, 1), "frac_of_peak": round(a2a_bytes / a2a_us / 1e3 / peak_gbs, 4)}
@@ -490,7 +504,7 @@ def run_gpu(args):
         "launches_since_load": int(launches_total),
         "device_status": status,
         "clocks": clocks,
-        "sweep": sweep, "allgather16": ag_row, "alltoall8": a2a_row, "decode_chain": chain_rows,
+        "sweep": sweep, "allgather16": ag_row, "alltoall8": a2a_row, "reduce_scatter8": rs_rows, "decode_chain": chain_rows,
     }
     line.update(extras)
     if cpu is not None:

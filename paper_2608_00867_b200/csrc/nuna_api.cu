@@ -754,6 +754,7 @@ int nuna_shutdown(void)
     if (c->staging) cudaFree(c->staging);
     if (c->stream) cudaStreamDestroy(c->stream);
     for (auto& kv : c->sm_plans) cudaFree(kv.second.base);
+    for (unsigned* d : c->retired_plans) cudaFree(d);
     delete c;
     g_ctx[dev] = nullptr;
     return NUNA_OK;

@@ -45,6 +45,7 @@ struct Context {
     nuna_topology_t topology = {};       // last probe result (have_topology says whether it is valid)
     bool have_topology = false;
     std::map<std::tuple<int, size_t, int>, SmPlan> sm_plans;
+    std::vector<unsigned*> retired_plans; // plans of an earlier topology, freed at shutdown
     std::mutex mutex;
 };
 

@@ -430,6 +430,10 @@ int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
         std::lock_guard<std::mutex> lock(c->mutex);
         c->topology = *out;
         c->have_topology = true;
+        // work lists planned under the previous topology are stale: retire them (kept allocated until
+        // shutdown, because captured graphs may still name them) and rebuild on the next call of each shape
+        for (auto& kv : c->sm_plans) c->retired_plans.push_back(kv.second.base);
+        c->sm_plans.clear();
     }
 
 done:
