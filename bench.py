@@ -368,6 +368,9 @@ def run_gpu(args):
             "oneshot_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=nb.NUNA_LAUNCH_PDL, stream=st)),
             "twoshot_put_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(
                 s, d, c, flags=nb.NUNA_TWOSHOT_PUT | nb.NUNA_LAUNCH_PDL, stream=st)),
+            # nuna_allreduce: the library picks the algorithm by size
+            "size_selected": lambda c: (lambda s, d, st: nb.nuna_allreduce(
+                s, d, c, flags=nb.NUNA_TWOSHOT_PUT | nb.NUNA_LAUNCH_PDL | nb.NUNA_PLACE_AUTO, stream=st)),
         }
         for wl in workloads.config_size_sweep(args.sweep_min, args.sweep_max):
             c, B = wl.count, wl.bytes_per_rank

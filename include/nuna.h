@@ -213,6 +213,14 @@ int nuna_allreduce_oneshot(const void* const* src, void* const* dst, int nranks,
 int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
                            size_t count, int dtype, unsigned flags, void* stream);
 
+/* Allreduce with the algorithm chosen by message size -- the counterpart of the paper's per-collective
+ * choice between routing schemes by a size threshold (Section 4.1.2): one-shot while the message is small
+ * enough for its single step to win (up to 128 KiB per rank, measured), the two-shot put form beyond.
+ * With NUNA_TWOSHOT_PUT clear in `flags` the large-message choice is the flag-barrier two-shot instead
+ * (set NUNA_TWOSHOT_PUT to allow the put form).  Same bits whichever is chosen.                          */
+int nuna_allreduce(const void* const* src, void* const* dst, int nranks,
+                   size_t count, int dtype, unsigned flags, void* stream);
+
 /* Reduce-scatter: src[k] holds nranks*shard_count elements, dst[r] holds shard_count elements;
  * dst[r][j] = fold over k of src[k][r*shard_count + j].                                               */
 int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks,

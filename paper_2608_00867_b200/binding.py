@@ -92,7 +92,7 @@ def lib() -> ctypes.CDLL:
         L = ctypes.CDLL(_LIB_PATH)
         vpp = ctypes.POINTER(ctypes.c_void_p)
         coll = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint, ctypes.c_void_p]
-        for name in ("nuna_allreduce_oneshot", "nuna_allreduce_twoshot", "nuna_reduce_scatter", "nuna_allgather",
+        for name in ("nuna_allreduce", "nuna_allreduce_oneshot", "nuna_allreduce_twoshot", "nuna_reduce_scatter", "nuna_allgather",
                      "nuna_alltoall"):
             getattr(L, name).argtypes = coll
             getattr(L, name).restype = ctypes.c_int
@@ -185,6 +185,10 @@ def nuna_set_option(option: int, value: int, check: bool = True) -> int:
 
 def nuna_allreduce_oneshot(src, dst, count, dtype=NUNA_BF16, flags=0, stream=None, check=True, nranks=None) -> int:
     return _collective("nuna_allreduce_oneshot", src, dst, count, dtype, flags, stream, check, nranks)
+
+
+def nuna_allreduce(src, dst, count, dtype=NUNA_BF16, flags=0, stream=None, check=True, nranks=None) -> int:
+    return _collective("nuna_allreduce", src, dst, count, dtype, flags, stream, check, nranks)
 
 
 def nuna_allreduce_twoshot(src, dst, count, dtype=NUNA_BF16, flags=0, stream=None, check=True, nranks=None) -> int:

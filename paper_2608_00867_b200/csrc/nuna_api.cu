@@ -620,6 +620,16 @@ int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
     return launch_twoshot(c, make_ptrs(src, dst, nranks), nranks, dtype, count, flags, (cudaStream_t)stream);
 }
 
+int nuna_allreduce(const void* const* src, void* const* dst, int nranks, size_t count, int dtype, unsigned flags,
+                   void* stream)
+{
+    // crossover measured on B200 at 8 ranks (cold and L2-resident): one-shot wins up to 128 KiB per rank
+    const size_t bytes = count * elem_size(dtype);
+    if (nranks <= 1 || bytes <= ((size_t)128 << 10))
+        return nuna_allreduce_oneshot(src, dst, nranks, count, dtype, flags & ~NUNA_TWOSHOT_PUT, stream);
+    return nuna_allreduce_twoshot(src, dst, nranks, count, dtype, flags, stream);
+}
+
 int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks, size_t shard_count, int dtype,
                         unsigned flags, void* stream)
 {

@@ -396,6 +396,17 @@ def test_two_host_threads_on_their_own_streams():
     assert not errors, errors
 
 
+def test_size_selected_allreduce_matches_oracle_on_both_sides_of_the_threshold():
+    for count in (1000, 64 * 1024, 64 * 1024 + 8, 300000):
+        for flags in (0, nb.NUNA_TWOSHOT_PUT, nb.NUNA_TWOSHOT_PUT | nb.NUNA_LAUNCH_PDL | nb.NUNA_PLACE_AUTO):
+            src = workloads.special_values(8, count, seed=count)
+            want = oracle.allreduce(src, nthreads=4)[0]
+            dst = Dst(8, count)
+            nb.nuna_allreduce(upload(src), dst.view, count, flags=flags)
+            for got in dst.numpy():
+                assert_same_bits(got, want, f"auto count={count} flags={flags}")
+
+
 def test_host_buffer_entry_point():
     for n, count, two in ((8, 32 * 8192, False), (8, 32 * 8192, True), (3, 1001, False), (3, 1001, True)):
         src = workloads.rank_buffers(n, count, "normal", seed=77)
