@@ -251,7 +251,7 @@ int nuna_alltoall(const void* const* src, void* const* dst, int nranks,
  *    many of binary32); larger messages return NUNA_ERR_TOO_LARGE and print the limit.  The array
  *    costs 4 MiB of device memory on every GPU that loads the library, for the life of the process.
  *  - The first call on a device looks up the array's device address and zeroes the barrier words
- *    (a synchronous 16-byte cudaMemset); make that first call before starting any stream capture.
+ *    (a small synchronous cudaMemset); make that first call before starting any stream capture.
  *  - All calls on a device share the one array, which keeps the previous call's shard; the kernel
  *    overwrites every element it later reads, so stale contents never reach a result.  Two calls that
  *    overlap on the GPU (different streams, no ordering) race on it: keep calls stream-ordered.

@@ -814,7 +814,7 @@ int nuna_debug_barrier_selftest(unsigned grid, unsigned expected, unsigned timeo
 //
 // Everything the flag-barrier two-shot needs beyond its inputs and outputs -- the shard
 // intermediate and the barrier words -- lives in the two file-scope device arrays below, which
-// every GPU that loads this library carries from module load to process exit (4 MiB + 16 bytes).
+// every GPU that loads this library carries from module load to process exit (4 MiB + 384 bytes).
 // In host code the names `g_static_shard` and `g_static_barrier` are only stand-ins for the
 // symbols, not device addresses; the addresses a kernel can use come from cudaGetSymbolAddress,
 // looked up once per device, with that device current, on the entry point's first call there.

@@ -16,11 +16,13 @@ struct RankPtrs {
 
 // Flag-barrier words and the latched device status, in device memory.
 struct BarrierWords {
-    unsigned int arrive;
-    unsigned int epoch;
+    unsigned int arrive;      // arrivals of the current round (atomics land here)
+    unsigned int pad0[31];
+    unsigned int epoch;       // bumped by the last arriver; polled by everyone else -- on its own 128-byte
+    unsigned int pad1[31];    // line so that the polling loads do not queue behind the arrival atomics
     unsigned int status;
     unsigned int work[2];     // dynamic work cursors of the fused two-shot's two phases (zero between launches)
-    unsigned int pad[3];
+    unsigned int pad2[29];
 };
 
 }  // namespace nuna
