@@ -265,7 +265,9 @@ int nuna_allreduce_twoshot_static(const void* const* src, void* const* dst, int 
 /* End-to-end variant with HOST buffers: src[r] / dst[d] are HOST pointers to `count` elements (pinned
  * or pageable).  Copies the sources to library-owned device staging buffers, runs the one-shot
  * (two_shot == 0) or two-shot allreduce, copies every destination back and synchronises.  Allocates
- * staging on first use or growth.                                                                       */
+ * staging on first use or growth.  With two_shot != 0 and NUNA_TWOSHOT_PUT, and every buffer page-locked
+ * (cudaHostAlloc / cudaHostRegister) and 16-byte aligned, the kernel works on the host buffers in place
+ * instead: every byte crosses the host link once, in both directions at the same time, with no copies.   */
 int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks,
                         size_t count, int dtype, unsigned flags, int two_shot);
 

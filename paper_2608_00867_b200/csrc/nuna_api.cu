@@ -682,6 +682,34 @@ int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks, si
     if ((st = get_context(&c)) != NUNA_OK) return st;
     std::lock_guard<std::mutex> lock(c->mutex);
     const size_t bytes = count * elem_size(dtype);
+    if (!c->stream && cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking) != cudaSuccess) return NUNA_ERR_CUDA;
+
+    // Page-locked host buffers are visible to the device: the put form of the two-shot reads every source
+    // byte once and writes every destination byte once, so it can run directly on them -- one kernel, reads
+    // and writes crossing the host link in both directions at once, no staging copies.
+    if (two_shot && (flags & NUNA_TWOSHOT_PUT)) {
+        const void* msrc[NUNA_MAX_RANKS];
+        void* mdst[NUNA_MAX_RANKS];
+        bool mapped = true;
+        for (int r = 0; r < nranks && mapped; ++r) {
+            cudaPointerAttributes as, ad;
+            if (cudaPointerGetAttributes(&as, src[r]) != cudaSuccess || cudaPointerGetAttributes(&ad, dst[r]) != cudaSuccess) {
+                cudaGetLastError();
+                mapped = false;
+                break;
+            }
+            mapped = as.type == cudaMemoryTypeHost && ad.type == cudaMemoryTypeHost && as.devicePointer && ad.devicePointer &&
+                     (((uintptr_t)as.devicePointer | (uintptr_t)ad.devicePointer) & 15u) == 0;
+            msrc[r] = as.devicePointer;
+            mdst[r] = ad.devicePointer;
+        }
+        if (mapped) {
+            st = launch_twoshot(c, make_ptrs(msrc, mdst, nranks), nranks, dtype, count, flags & ~NUNA_LAUNCH_PDL, c->stream);
+            if (st != NUNA_OK) return st;
+            return cudaStreamSynchronize(c->stream) == cudaSuccess ? NUNA_OK : NUNA_ERR_CUDA;
+        }
+    }
+
     const size_t slot = (bytes + 255) & ~(size_t)255;
     const size_t need = slot * 2 * (size_t)nranks;
     if (need > c->staging_bytes) {
@@ -691,7 +719,6 @@ int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks, si
         if (cudaMalloc(&c->staging, need) != cudaSuccess) return NUNA_ERR_CUDA;
         c->staging_bytes = need;
     }
-    if (!c->stream && cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking) != cudaSuccess) return NUNA_ERR_CUDA;
     if (two_shot && !(flags & NUNA_TWOSHOT_PUT) && (st = ensure_scratch(c, slot)) != NUNA_OK) return st;
     const void* dsrc[NUNA_MAX_RANKS];
     void* ddst[NUNA_MAX_RANKS];

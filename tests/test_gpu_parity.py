@@ -417,6 +417,24 @@ def test_host_buffer_entry_point():
             assert np.array_equal(dst[d], want)
 
 
+def test_host_entry_point_in_place_on_pinned_buffers():
+    for n, count in ((8, 32 * 8192), (3, 1001), (16, 4096)):
+        src = workloads.special_values(n, count, seed=5 + n)
+        want = oracle.allreduce(src, nthreads=4)[0]
+        psrc = [torch.from_numpy(a.view(np.int16).copy()).pin_memory() for a in src]
+        pdst = [torch.zeros(count, dtype=torch.int16).pin_memory() for _ in range(n)]
+        before = nb.nuna_launch_count()
+        nb.nuna_allreduce_host(psrc, pdst, count, flags=nb.NUNA_TWOSHOT_PUT, two_shot=True)
+        assert nb.nuna_launch_count() == before + 1
+        for t in pdst:
+            assert_same_bits(t.numpy().view(np.uint16), want, "pinned in place")
+        # pageable destinations fall back to staging copies, same bits
+        hdst = [np.zeros(count, dtype=np.uint16) for _ in range(n)]
+        nb.nuna_allreduce_host(psrc, hdst, count, flags=nb.NUNA_TWOSHOT_PUT, two_shot=True)
+        for h in hdst:
+            assert_same_bits(h, want, "pageable fallback")
+
+
 def test_argument_errors_launch_nothing():
     a = [torch.zeros(64, dtype=torch.int16, device="cuda") for _ in range(2)]
     b = [torch.zeros(64, dtype=torch.int16, device="cuda") for _ in range(2)]
