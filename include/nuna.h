@@ -90,6 +90,11 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
  * first call for a given (nranks, count) builds and uploads the plan (allocates: NUNA_ERR_CAPTURING on a
  * capturing stream); later calls only launch.  Calls sharing a plan must be stream-ordered.             */
 #define NUNA_PLACE_SM_LISTS   128u
+/* `flags`, bit 8, with NUNA_PLACE_AWARE on nuna_allreduce_oneshot, 2 <= nranks <= 8: run each tile's N work
+ * items as one thread-block cluster of N blocks (placed by the hardware on one GPC).  Block r fetches
+ * source r's tile once into shared memory; after a cluster barrier every block reads all N tiles from its
+ * neighbours' shared memory and folds them for its own destination.  Ignored for other rank counts.     */
+#define NUNA_PLACE_CLUSTER    256u
 
 /* ---- topology probe --------------------------------------------------------------------------------
  * Result of nuna_probe_topology: caller-owned, plain data, fixed maximum sizes.  Latencies are in SM

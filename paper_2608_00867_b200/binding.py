@@ -29,6 +29,7 @@ NUNA_TWOSHOT_PUT = 16
 NUNA_HINT_RESIDENT = 32
 NUNA_LAUNCH_PDL = 64
 NUNA_PLACE_SM_LISTS = 128
+NUNA_PLACE_CLUSTER = 256
 
 NUNA_MAX_SMS, NUNA_MAX_PROBE_BUFS, NUNA_PROBE_REGIONS, NUNA_MAX_PROBE_LINES = 256, 32, 8, 2048
 NUNA_TOPO_UNIFORM, NUNA_TOPO_NONUNIFORM = 0, 1

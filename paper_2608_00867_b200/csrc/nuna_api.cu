@@ -83,7 +83,8 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
     if (nranks > NUNA_MAX_RANKS) return NUNA_ERR_TOO_MANY_RANKS;
     if (nranks < 1) return NUNA_ERR_INVALID_ARG;
     if (dtype != NUNA_BF16 && dtype != NUNA_F16 && dtype != NUNA_F32) return NUNA_ERR_UNSUPPORTED_DTYPE;
-    if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT | NUNA_HINT_RESIDENT | NUNA_LAUNCH_PDL | NUNA_PLACE_SM_LISTS)) != 0u ||
+    if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT | NUNA_HINT_RESIDENT | NUNA_LAUNCH_PDL | NUNA_PLACE_SM_LISTS |
+                   NUNA_PLACE_CLUSTER)) != 0u ||
         (flags & NUNA_PLACE_MASK) == 3u)
         return NUNA_ERR_INVALID_ARG;
     if (src_elems > ((size_t)1 << 40) || dst_elems > ((size_t)1 << 40)) return NUNA_ERR_TOO_LARGE;
@@ -162,6 +163,8 @@ static unsigned launch_mode(unsigned flags, size_t total_src_bytes = 0)
     return ((flags & NUNA_LAUNCH_PDL) && total_src_bytes <= ((size_t)16 << 20)) ? kLaunchPdl : kLaunchPlain;
 }
 
+static thread_local unsigned t_cluster_dim = 0;           // > 0: next launch() uses clusters of this many blocks
+
 template <typename... Args, typename... Act>
 static int launch(void (*kernel)(Args...), unsigned grid, cudaStream_t stream, unsigned mode, Act&&... args)
 {
@@ -170,8 +173,16 @@ static int launch(void (*kernel)(Args...), unsigned grid, cudaStream_t stream, u
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[3];
     int nattr = 0;
+    if (t_cluster_dim > 0) {
+        attr[nattr].id = cudaLaunchAttributeClusterDimension;
+        attr[nattr].val.clusterDim.x = t_cluster_dim;
+        attr[nattr].val.clusterDim.y = 1;
+        attr[nattr].val.clusterDim.z = 1;
+        ++nattr;
+        t_cluster_dim = 0;
+    }
     if (mode & kLaunchCooperative) {
         attr[nattr].id = cudaLaunchAttributeCooperative;
         attr[nattr].val.cooperative = 1;
@@ -404,6 +415,18 @@ static int launch_sm_lists(Context* c, const RankPtrs& p, size_t count, unsigned
     return launch(k, grid, stream, mode, p, count, sl, blocks_per_sm);
 }
 
+template <int N, int DT>
+static int launch_cluster(Context* c, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
+{
+    auto k = k_oneshot_cluster<N, DT>;
+    const size_t nvec = count / Elem<DT>::kElems;
+    const size_t ntiles = std::max<size_t>(1, ceil_div(nvec, (size_t)kThreads));
+    size_t clusters = std::min<size_t>(ntiles, (size_t)1 << 20);
+    if (c->blocks_override > 0) clusters = std::max<size_t>(1, std::min<size_t>(clusters, (size_t)c->blocks_override / N));
+    t_cluster_dim = N;
+    return launch(k, (unsigned)(clusters * N), stream, mode, p, count, ntiles);
+}
+
 template <int N, int C, int DT>
 static int launch_group(Context* c, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
 {
@@ -426,6 +449,13 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
     if (place == NUNA_PLACE_AWARE || (place == NUNA_PLACE_AUTO && aware_pays_off(c, nranks, bytes, flags))) {
         // co-location factor: C destinations of a tile share a block (C <= N rounded up to a power of two)
         const int coloc = coloc_for(c, nranks);
+        if ((flags & NUNA_PLACE_CLUSTER) && nranks >= 2 && nranks <= 8) {
+            return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
+                constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
+                if constexpr (N >= 2 && N <= 8) return launch_cluster<N, DT>(c, p, count, mode, stream);
+                else return NUNA_ERR_INVALID_ARG;
+            });
+        }
         if (flags & NUNA_PLACE_SM_LISTS) {
             return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
                 constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;

@@ -314,6 +314,70 @@ k_oneshot_group(const RankPtrs p, const size_t count, const size_t ntiles)
     }
 }
 
+// ---- one-shot allreduce, a logical group per thread-block cluster --------------------------------------
+//
+// The hardware's own locality domain is the GPC: the blocks of a thread-block cluster are placed on
+// one GPC and can read each other's shared memory.  Here the N work items (tile, d) of one tile --
+// one logical group of Section 4.2.1 -- form one cluster of N blocks.  Block r first loads source
+// r's tile, one 16-byte vector per thread, into its shared memory: the cluster as a whole fetches
+// every source byte exactly once, with all of its loads in flight at the same time.  After a
+// cluster barrier, block d (emulated rank d) reads the N source tiles out of the N blocks' shared
+// memories (ld.shared::cluster), folds them in rank order and stores its own destination.  Each
+// emulated rank still does its own N reads and its own fold; the reads are served by the
+// neighbours' shared memory instead of L2.  Few registers are live, so all groups of a mid-sized
+// message are resident at once (no second wave).
+__device__ __forceinline__ unsigned cluster_ctarank()
+{
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ uint4 ld_dsmem(const uint4* local_ptr, unsigned cta)
+{
+    unsigned local = (unsigned)__cvta_generic_to_shared(local_ptr), remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(cta));
+    uint4 v;
+    asm volatile("ld.shared::cluster.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(remote) : "memory");
+    return v;
+}
+
+template <int N, int DT>
+__global__ void __launch_bounds__(kThreads)
+k_oneshot_cluster(const RankPtrs p, const size_t count, const size_t ntiles)
+{
+    pdl_wait();
+    __shared__ __align__(16) uint4 tile[kThreads];
+    const unsigned r = cluster_ctarank();                  // this block's source to fetch and destination to write
+    const size_t nvec = count / Elem<DT>::kElems;
+    const size_t nclusters = gridDim.x / N, cluster_id = blockIdx.x / N;
+    for (size_t t = cluster_id; t < ntiles; t += nclusters) {
+        const size_t i = t * kThreads + threadIdx.x;
+        if (i < nvec) tile[threadIdx.x] = ld_src(p.src[r] + i);
+        cluster_sync();                                    // every block's tile is in its shared memory
+        if (i < nvec) {
+            uint4 v[N];
+#pragma unroll
+            for (int s = 0; s < N; ++s) v[s] = ld_dsmem(&tile[threadIdx.x], (unsigned)s);
+            st_dst(p.dst[r] + i, fold_vectors<N, DT>(v));
+        }
+        cluster_sync();                                    // nobody still reads a tile that is about to be replaced
+    }
+    pdl_trigger();
+    const size_t tail0 = nvec * Elem<DT>::kElems;
+    if (tail0 < count && cluster_id == 0) {
+        const size_t e = tail0 + threadIdx.x;
+        if (e < count) store_elem<DT>(p.dst[r], e, fold_scalar<N, DT>(p, e));
+    }
+}
+
 // ---- one-shot allreduce through per-SM work lists (the planner's M_compute at SM granularity) ------------
 //
 // CUDA has no thread-block -> SM affinity mask (the paper's dispatcher mechanism, Section 4.2.3), so

@@ -44,6 +44,8 @@ def assert_same_bits(got, want, dtype, what):
 ALGOS = {
     "oneshot": lambda s, d, c, dt: nb.nuna_allreduce_oneshot(s, d, c, dtype=dt),
     "oneshot_aware": lambda s, d, c, dt: nb.nuna_allreduce_oneshot(s, d, c, dtype=dt, flags=nb.NUNA_PLACE_AWARE),
+    "oneshot_cluster": lambda s, d, c, dt: nb.nuna_allreduce_oneshot(s, d, c, dtype=dt,
+                                                                    flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_CLUSTER),
     "oneshot_sm_lists": lambda s, d, c, dt: nb.nuna_allreduce_oneshot(s, d, c, dtype=dt,
                                                                      flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS),
     "twoshot": lambda s, d, c, dt: nb.nuna_allreduce_twoshot(s, d, c, dtype=dt),

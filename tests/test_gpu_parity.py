@@ -58,7 +58,7 @@ COUNTS = [1, 7, 8, 9, 15, 16, 17, 2047, 2048, 2049, 4096, 6151, 100003, 262144]
 
 
 @pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16])
-@pytest.mark.parametrize("algo", ["oneshot", "oneshot_aware", "oneshot_sm_lists", "twoshot", "twoshot_put"])
+@pytest.mark.parametrize("algo", ["oneshot", "oneshot_aware", "oneshot_cluster", "oneshot_sm_lists", "twoshot", "twoshot_put"])
 def test_allreduce_special_values_all_counts(n, algo):
     for count in COUNTS:
         src = workloads.special_values(n, count, seed=1000 * n + count % 997)
@@ -68,6 +68,8 @@ def test_allreduce_special_values_all_counts(n, algo):
             nb.nuna_allreduce_oneshot(dsrc, dst.view, count)
         elif algo == "oneshot_aware":
             nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE)
+        elif algo == "oneshot_cluster":
+            nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_CLUSTER)
         elif algo == "oneshot_sm_lists":
             nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS)
         else:
@@ -164,6 +166,7 @@ def test_sweep_sizes_one_and_two_shot_agree_with_oracle():
         want = oracle.allreduce(src, nthreads=8)[0]
         dsrc = upload(src)
         for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE),
+                            (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_CLUSTER | nb.NUNA_LAUNCH_PDL),
                             (nb.nuna_allreduce_twoshot, 0), (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
             dst = Dst(w.nranks, w.count)
             call(dsrc, dst.view, w.count, flags=flags)
@@ -192,6 +195,7 @@ def test_full_size_64MiB_sampled_columns_and_invariants():
     want = oracle.allreduce([np.ascontiguousarray(c) for c in cols], nthreads=4)[0]
     results = []
     for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE),
+                        (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_CLUSTER),
                         (nb.nuna_allreduce_twoshot, 0), (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
         dst = [torch.full((count,), -1, dtype=torch.int16, device="cuda") for _ in range(n)]
         call(dsrc, dst, count, flags=flags)
