@@ -284,6 +284,7 @@ def run_gpu(args):
     }
     place = {}
     for pname, pflags in (("roundrobin", nb.NUNA_PLACE_ROUNDROBIN), ("aware_colocated", nb.NUNA_PLACE_AWARE),
+                          ("aware_cluster_dsmem", nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_CLUSTER),
                           ("aware_sm_lists", nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS)):
         fn = lambda s, d, st, f=pflags: nb.nuna_allreduce_oneshot(s, d, count, flags=f, stream=st)
         place[pname] = {"cold_us": round(per_call_us(fn, sets, 1000, 3), 3),
