@@ -363,6 +363,31 @@ def test_tuning_options_change_the_launch_not_the_bits():
     assert nb.nuna_device_status() == nb.NUNA_OK
 
 
+def test_minimum_alignment_sixteen_bytes_only():
+    """Buffers that are 16-byte aligned but not 32-, 64- or 128-byte aligned, each rank at a different offset."""
+    n, count = 8, 20011
+    src = workloads.special_values(n, count, seed=61)
+    want = oracle.allreduce(src, nthreads=4)[0]
+    pad = 8 * 16
+    big_s = [torch.zeros(count + pad, dtype=torch.int16, device="cuda") for _ in range(n)]
+    big_d = [torch.zeros(count + pad, dtype=torch.int16, device="cuda") for _ in range(n)]
+    dsrc, ddst = [], []
+    for r in range(n):
+        off = 8 * (2 * r + 1)                                   # odd multiples of 16 bytes
+        big_s[r][off:off + count] = torch.from_numpy(src[r].view(np.int16)).cuda()
+        dsrc.append(big_s[r][off:off + count])
+        ddst.append(big_d[r][8 * (2 * (n - r) - 1): 8 * (2 * (n - r) - 1) + count])
+        assert dsrc[-1].data_ptr() % 32 == 16 and ddst[-1].data_ptr() % 32 == 16
+    for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE),
+                        (nb.nuna_allreduce_twoshot, 0), (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
+        for t in big_d:
+            t.zero_()
+        call(dsrc, ddst, count, flags=flags)
+        torch.cuda.synchronize()
+        for t in ddst:
+            assert_same_bits(t.cpu().numpy().view(np.uint16), want, f"{call.__name__} {flags}")
+
+
 def test_two_host_threads_on_their_own_streams():
     """Calls that share no library state (one-shot, two-shot put, allgather) may be issued from
     different host threads on different streams at the same time."""
