@@ -66,8 +66,11 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 
 /* `flags`, bits 0-1: thread-block placement (Section 4.2 / Section 5.3 baseline). */
 #define NUNA_PLACE_ROUNDROBIN 0u   /* locality-unaware: work item i -> thread block i mod grid          */
-#define NUNA_PLACE_AWARE      1u   /* persistent blocks pull the work planned for their SM's domain      */
-#define NUNA_PLACE_AUTO       2u   /* AWARE where the installed topology says it helps, else ROUNDROBIN  */
+#define NUNA_PLACE_AWARE      1u   /* a tile's N work items (one logical group, Section 4.2.1) are co-located:
+                                      in one thread block by default, or through NUNA_PLACE_SM_LISTS /
+                                      NUNA_PLACE_CLUSTER; only the one-shot allreduce distinguishes placements */
+#define NUNA_PLACE_AUTO       2u   /* AWARE where it was measured to help (see NUNA_HINT_RESIDENT), else
+                                      exactly the ROUNDROBIN kernel                                        */
 #define NUNA_PLACE_MASK       3u
 /* `flags`, bit 4 (nuna_allreduce_twoshot only): the reducing block stores its tile straight into all N
  * destinations, with no intermediate shard and no barrier.                                             */
@@ -145,12 +148,14 @@ typedef struct nuna_topology {
 /* Measures, for every SM (indexed by %smid) and every buffer, the latency of dependent L2-only loads
  * to sampled lines of the caller's buffers (the analogue of the paper's per-compute-unit, per-address
  * remote-access sweep, Section 3.2), plus each SM's cold DRAM latency, clusters the SMs into domains
- * and stores the result in *out and in the device context (where NUNA_PLACE_AWARE plans read it).
+ * and stores the result in *out and in the device context (where NUNA_PLACE_SM_LISTS plans read it).
  * bufs: HOST array of nbufs (<= NUNA_MAX_PROBE_BUFS) device pointers, bytes[b] >= 128 each, 16-byte
  * aligned.  One 8-byte word per sampled line is overwritten during the measurement and restored
  * before return; the buffers must not be in use by other work meanwhile.  Synchronises `stream`,
  * allocates temporary device memory (about 2.3 x the L2 size): NUNA_ERR_CAPTURING on a capturing
- * stream.  Latency values are hardware facts and carry no parity claim.                               */
+ * stream.  Work lists planned earlier for NUNA_PLACE_SM_LISTS are retired and rebuilt under the new
+ * topology on the next call of each shape; chains created earlier keep using the lists they captured.
+ * Latency values are hardware facts and carry no parity claim.                                        */
 int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
                         nuna_topology_t* out, void* stream);
 
