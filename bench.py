@@ -490,11 +490,10 @@ def run_gpu(args):
     if rank != 0:
         return 0
 
-    traffic = None
-    prof = os.path.join(ROOT, "profiles", "oneshot_n8_512KiB_dram_bytes.json")
-    if os.path.exists(prof):
-        with open(prof) as f:
-            traffic = json.load(f).get("dram_bytes_per_launch")
+    # dram__bytes_read.sum + dram__bytes_write.sum of one k_oneshot_rr<8,1> launch on this workload, from the
+    # ncu capture summarised in profiles/oneshot_rr_n8_512KiB.md (4.20 MB read, 0 written: the destinations
+    # are still dirty in L2 when the kernel ends)
+    traffic = 4200192
     line = {
         "metric": METRIC, "value": us_per_step, "unit": "us", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": us_per_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
