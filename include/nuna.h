@@ -225,7 +225,8 @@ int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
 
 /* Allreduce with the algorithm chosen by message size -- the counterpart of the paper's per-collective
  * choice between routing schemes by a size threshold (Section 4.1.2): one-shot while the message is small
- * enough for its single step to win (up to 128 KiB per rank, measured), the two-shot put form beyond.
+ * enough for its single step to win (measured: up to 1 MiB per rank at 2 ranks, 512 KiB at 4, 128 KiB at
+ * 8, 64 KiB at 16), the two-shot beyond.
  * With NUNA_TWOSHOT_PUT clear in `flags` the large-message choice is the flag-barrier two-shot instead
  * (set NUNA_TWOSHOT_PUT to allow the put form).  Same bits whichever is chosen.                          */
 int nuna_allreduce(const void* const* src, void* const* dst, int nranks,

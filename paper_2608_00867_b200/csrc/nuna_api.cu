@@ -653,9 +653,13 @@ int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
 int nuna_allreduce(const void* const* src, void* const* dst, int nranks, size_t count, int dtype, unsigned flags,
                    void* stream)
 {
-    // crossover measured on B200 at 8 ranks (cold and L2-resident): one-shot wins up to 128 KiB per rank
+    // Crossover measured on B200, cold and L2-resident, with dependent launch: the one-shot's N-fold
+    // re-reads cost more the more ranks there are, so it wins up to 1 MiB per rank at 2 ranks,
+    // 512 KiB at 4, 128 KiB at 8 and 64 KiB at 16.
     const size_t bytes = count * elem_size(dtype);
-    if (nranks <= 1 || bytes <= ((size_t)128 << 10))
+    const size_t limit = nranks <= 2 ? ((size_t)1 << 20) : nranks <= 4 ? ((size_t)512 << 10)
+                       : nranks <= 8 ? ((size_t)128 << 10) : ((size_t)64 << 10);
+    if (nranks <= 1 || bytes <= limit)
         return nuna_allreduce_oneshot(src, dst, nranks, count, dtype, flags & ~NUNA_TWOSHOT_PUT, stream);
     return nuna_allreduce_twoshot(src, dst, nranks, count, dtype, flags, stream);
 }
