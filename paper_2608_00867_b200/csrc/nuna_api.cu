@@ -117,11 +117,13 @@ static RankPtrs make_ptrs(const void* const* src, void* const* dst, int nranks)
 
 // ---- launch configuration --------------------------------------------------------------------
 
-// Vectors per thread per item.  Chosen so a thread keeps about 8-16 independent 16-byte loads in
-// flight whatever N is, without pushing register use past two or three blocks per SM.
+// Vectors per thread per item.  One: with one work item per block and N independent 16-byte loads in
+// flight per thread, more vectors per thread only mean fewer blocks (measured at 2 and 4 ranks: 64 KiB
+// per rank 1.43 us with one vector, 1.64 us with four; no difference at 16 MiB).  NUNA_OPT_UNROLL
+// overrides it for experiments.
 static int pick_unroll(const Context* c, int nranks)
 {
-    int u = nranks >= 8 ? 1 : nranks >= 4 ? 2 : 4;
+    int u = 1;
     if (c->unroll_override == 1 || c->unroll_override == 2 || c->unroll_override == 4) u = c->unroll_override;
     while (u > 1 && u * nranks > 16) u >>= 1;
     return u;
@@ -932,7 +934,7 @@ extern "C" int nuna_allreduce_twoshot_static(const void* const* src, void* const
     }
     StaticSetup* s = nullptr;
     if ((st = static_setup(&s)) != NUNA_OK) return st;
-    const int u = nranks >= 8 ? 1 : nranks >= 4 ? 2 : 4;
+    const int u = 1;
     return launch_twoshot_fused(s->num_sms, 0, make_ptrs(src, dst, nranks), nranks, dtype, count, u, s->shard, s->barrier,
                                 1000000000ull, (cudaStream_t)stream);
 }
