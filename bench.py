@@ -3,16 +3,20 @@
 
 A *step* is one one-shot allreduce over 8 emulated ranks of 512 KiB each (batch 32 x
 hidden 8192 bf16 per rank, N(0,1), the tensor-parallel decode activation), issued through
-the C ABI.  The K timed steps are captured in a CUDA graph (the way a decode step issues
-its collectives) that rotates over enough buffer sets to exceed twice the L2 capacity, so
-every step reads its sources from HBM ("cold").  Timing is by CUDA events on the launching
-stream; with N GPUs each rank runs an independent replica (the emulation has no inter-GPU
-step) and the slowest rank's time is used.
+the C ABI.  The K steps are the nodes of one CUDA graph (the way a decode step issues its
+collectives) that rotates over enough buffer sets to exceed twice the L2 capacity, so every
+step reads its sources from HBM ("cold").  One pass of the K steps is one sample; passes are
+repeated back to back until the timed region is at least 50 ms long, each pass with its own
+CUDA events on the launching stream, and the reported value is the median pass divided by K.
+With N GPUs each rank runs an independent replica (the emulation has no inter-GPU step) and
+the slowest rank's time is used.
 
-Besides the headline the JSON line carries, per message size (8 KiB ... 64 MiB per rank),
-the latency and algorithmic HBM throughput of one-shot, two-shot (flag barrier) and
-two-shot-put, cold and warm; the 16-rank allgather; the launch floor; the 160-node decode
-chain; the oracle timed on the host cores; and an end-to-end number with host buffers.
+Output: every detail section (message-size sweep 8 KiB ... 64 MiB per rank with one-shot,
+two-shot and put variants, cold and warm, isolated per-call latencies, launch floors, the
+16-rank allgather, reduce-scatter, alltoall, the 160-node decode chain, probe summary,
+placement, domain-count and block-count sensitivity, interference) is printed on its own
+stdout line as it completes and collected in gpurun_out/bench_detail.json; the LAST stdout
+line is the compact result object.
 """
 from __future__ import annotations
 
@@ -31,43 +35,106 @@ if ROOT not in sys.path:
 
 METRIC = "allreduce_latency_us"
 N_RANKS = 8
+MIN_TIMED_MS = 50.0
+DTYPE = "bf16 storage, f32 accumulate"
+
+
+def PLACEMENT_VARIANTS(nb):
+    """One-shot placements compared on the headline workload (flags of nuna_allreduce_oneshot)."""
+    A = nb.NUNA_PLACE_AWARE
+    return {"roundrobin": nb.NUNA_PLACE_ROUNDROBIN, "aware_colocated": A, "aware_staged": A | nb.NUNA_PLACE_STAGED,
+            "aware_cluster_dsmem": A | nb.NUNA_PLACE_CLUSTER, "aware_sm_lists": A | nb.NUNA_PLACE_SM_LISTS,
+            "auto": nb.NUNA_PLACE_AUTO, "auto_resident_hint": nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT}
+
+
+def CHAIN_VARIANTS(nb):
+    """Decode-chain variants (flags of nuna_chain_create): CUDA graph of one kernel per node, or one kernel."""
+    P, G = nb.NUNA_LAUNCH_PDL, nb.NUNA_CHAIN_GRAPH
+    return {"graph_roundrobin": G, "graph_roundrobin_pdl": G | P,
+            "graph_aware_pdl": G | nb.NUNA_PLACE_AWARE | P,
+            "graph_staged_pdl": G | nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_STAGED | nb.NUNA_HINT_RESIDENT | P,
+            "graph_auto_resident_pdl": G | nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT | P,
+            "graph_sm_lists_pdl": G | nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS | P,
+            "persistent_single_kernel": nb.NUNA_CHAIN_PERSISTENT,
+            "library_choice": nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT | P}
 
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
-    return 6650.0, "fallback (earlier measurement on this pool)"
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def recorded_traffic(kernel_key):
+    """DRAM bytes per launch of a kernel, as recorded from an ncu capture (profiles/dram_traffic.json)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f).get(kernel_key, {}).get("dram_bytes_per_launch")
+    except (OSError, ValueError):
+        return None
+
+
+def pctl(sorted_vals, q):
+    if not sorted_vals:
+        return None
+    i = min(len(sorted_vals) - 1, max(0, int(round(q * (len(sorted_vals) - 1)))))
+    return sorted_vals[i]
+
+
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def oracle_time(src, nthreads, seconds):
+    """The oracle as it stands, repeated for about `seconds` after a warm-up, in batches of 5 calls.
+    Returns (best batch, median batch) in us per allreduce and the number of calls.  The best batch is the
+    reported value: the host is shared, and interference only ever adds time."""
+    import oracle
+    t_end = time.perf_counter() + min(0.5, seconds / 3)
+    while time.perf_counter() < t_end:                           # thread pool, page faults, caches
+        oracle.allreduce(src, nthreads=nthreads)
+    per, calls, t_stop = [], 0, time.perf_counter() + seconds
+    while time.perf_counter() < t_stop or len(per) < 3:
+        t0 = time.perf_counter()
+        for _ in range(5):
+            oracle.allreduce(src, nthreads=nthreads)
+        per.append((time.perf_counter() - t0) / 5 * 1e6)
+        calls += 5
+    per.sort()
+    return per[0], pctl(per, 0.5), calls
+
+
+def cpu_baseline_block(src, workload_name):
+    cores = host_cores()
+    best, med, calls = oracle_time(src, cores, 3.0)
+    best1, med1, calls1 = oracle_time(src, 1, 1.5)
+    return {"value": round(best, 1), "unit": "us", "cores": cores, "kind": "oracle",
+            "sample": f"{calls} allreduces of {workload_name} in 3 s, best 5-call batch (median batch {med:.0f} us)",
+            "one_core_us": round(best1, 1)}
 
 
 # ---- reference arm: the CPU oracle ----------------------------------------------------------------
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return 0
-    import oracle
     from paper_2608_00867_b200 import workloads
     w = workloads.config_decode_activation()
-    src = workloads.make(w)
-    cores = os.cpu_count() or 1
-    for _ in range(max(args.warmup, 1)):
-        oracle.allreduce(src, nthreads=cores)
-    steps = max(1, min(args.steps, 2000))
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        oracle.allreduce(src, nthreads=cores)
-    dt = time.perf_counter() - t0
-    us = dt / steps * 1e6
+    cpu = cpu_baseline_block(workloads.make(w), w.name)
+    us = cpu["value"]
     line = {
         "impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus,
-        "steps": steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic",
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
         "config": {"workload": w.name, "nranks": w.nranks, "bytes_per_rank": w.bytes_per_rank,
-                   "algorithm": "oracle (plain C fold, OpenMP over elements)"},
-        "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle",
-                         "sample": f"{steps} whole allreduces of the 8 x 512 KiB workload"},
+                   "algorithm": "oracle (plain C fold, OpenMP over elements); a step = one allreduce"},
+        "cpu_baseline": cpu,
         "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -151,6 +218,13 @@ def run_gpu(args):
         sampler.start()
 
     barrier, max_over_ranks = rep.barrier, rep.max_over_ranks
+    detail = {}
+
+    def emit(name, obj):
+        """A finished detail section: kept for the detail file and printed on its own line by rank 0."""
+        detail[name] = obj
+        if rank == 0:
+            print(json.dumps({"detail": name, "data": obj}), flush=True)
 
     def make_sets(n, count, dst_count, min_bytes, dist_name="normal", seed=1, max_sets=4096):
         """Device buffer sets whose total footprint exceeds min_bytes (cold protocol).
@@ -188,45 +262,86 @@ def run_gpu(args):
                     fn(*sets[i % len(sets)], stream)
         return g
 
-    def time_graph(g, replays, warm_replays=1):
+    def time_passes(graphs, calls_per_pass, min_ms, min_passes, warm_passes=1, max_passes=20000):
+        """Replays the graph(s) of one pass back to back, every pass between its own pair of events, until the
+        timed region is at least min_ms long.  Returns per-call microseconds (slowest rank) of every pass and
+        the whole region's mean."""
         with torch.cuda.stream(stream):
-            for _ in range(warm_replays):
+            for _ in range(warm_passes):
+                for g in graphs:
+                    g.replay()
+            for g in graphs:                                         # first pass after a change of kernel: not representative
                 g.replay()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            barrier()
-            t0 = time.time()
-            e0.record(stream)
-            for _ in range(replays):
-                g.replay()
-            e1.record(stream)
-            barrier()
-            t1 = time.time()
-        sampler.mark(t0, t1)
-        return max_over_ranks(e0.elapsed_time(e1))                   # ms, slowest rank
-
-    def per_call_us(fn, sets, nodes, replays):
-        g = capture(fn, sets, nodes)
-        ms = time_graph(g, replays)
-        del g
-        return ms * 1e3 / (nodes * replays)
-
-    def per_call_stats(fn, sets, nodes, replays):
-        """Each replay of the graph timed on its own (its own event pair): median / min / max per call."""
-        g = capture(fn, sets, nodes)
-        with torch.cuda.stream(stream):
-            g.replay()
-            evs = [torch.cuda.Event(enable_timing=True) for _ in range(replays + 1)]
+            e = [torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)]
+            e[0].record(stream)
+            for _ in range(3):
+                for g in graphs:
+                    g.replay()
+            e[1].record(stream)
+            torch.cuda.synchronize()
+            est_ms = max(e[0].elapsed_time(e[1]) / 3, 1e-3)
+            passes = int(max(min_passes, min(max_passes, min_ms / est_ms * 1.25 + 1)))
+            if world > 1:
+                passes = int(max_over_ranks(passes))
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(passes + 1)]
             barrier()
             t0 = time.time()
             evs[0].record(stream)
-            for i in range(replays):
-                g.replay()
+            for i in range(passes):
+                for g in graphs:
+                    g.replay()
                 evs[i + 1].record(stream)
             barrier()
-            sampler.mark(t0, time.time())
-        per = sorted(max_over_ranks(evs[i].elapsed_time(evs[i + 1])) * 1e3 / nodes for i in range(replays))
+            t1 = time.time()
+        sampler.mark(t0, t1)
+        per = [max_over_ranks(evs[i].elapsed_time(evs[i + 1])) * 1e3 / calls_per_pass for i in range(passes)]
+        total_ms = max_over_ranks(evs[0].elapsed_time(evs[passes]))
+        return per, total_ms
+
+    def stats_of(per):
+        s = sorted(per)
+        return {"median": pctl(s, 0.5), "min": s[0], "p95": pctl(s, 0.95), "max": s[-1], "samples": len(s)}
+
+    def per_call_stats(fn, sets, nodes, min_ms=4.0, min_passes=20):
+        g = capture(fn, sets, nodes)
+        per, _ = time_passes([g], nodes, min_ms, min_passes)
         del g
-        return {"median": per[len(per) // 2], "min": per[0], "max": per[-1]}
+        return stats_of(per)
+
+    def per_call_us(fn, sets, nodes, min_ms=4.0, min_passes=5):
+        return per_call_stats(fn, sets, nodes, min_ms, min_passes)["median"]
+
+    def isolated_stats(fn, sets, reps=200):
+        """One eager call at a time: sync, event, call, event.  Median / p95 of `reps` (device time of a lone call,
+        launch included; the sets rotate, so with enough of them every call is cold)."""
+        per = []
+        with torch.cuda.stream(stream):
+            for i in range(10):
+                fn(*sets[i % len(sets)], stream)
+            torch.cuda.synchronize()
+            for i in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                fn(*sets[i % len(sets)], stream)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                per.append(e0.elapsed_time(e1) * 1e3)
+        s = sorted(per)
+        return {"median": round(pctl(s, 0.5), 3), "p95": round(pctl(s, 0.95), 3), "min": round(s[0], 3)}
+
+    def host_sync_floor(fn, sets, reps=300):
+        """Host clock around one eager call + cudaStreamSynchronize: what a caller that waits for the result pays."""
+        per = []
+        for i in range(20):
+            fn(*sets[i % len(sets)], stream)
+        stream.synchronize()
+        for i in range(reps):
+            t0 = time.perf_counter()
+            fn(*sets[i % len(sets)], stream)
+            stream.synchronize()
+            per.append((time.perf_counter() - t0) * 1e6)
+        s = sorted(per)
+        return {"median": round(pctl(s, 0.5), 3), "p95": round(pctl(s, 0.95), 3), "min": round(s[0], 3)}
 
     # ---- headline: K one-shot allreduces on the decode activation ------------------------------------
     w = workloads.config_decode_activation()
@@ -235,66 +350,90 @@ def run_gpu(args):
     headline_flags = nb.NUNA_PLACE_AUTO | nb.NUNA_LAUNCH_PDL
     oneshot = lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, count, flags=headline_flags, stream=st)
     K, W = args.steps, max(args.warmup, 3)
-    nodes = min(K, 1000)
-    replays, rem = divmod(K, nodes)
-    launches0 = nb.nuna_launch_count()
+    # The unit that is replayed and timed is a graph of m whole passes of K steps (m = 1000 // K when K is
+    # small, so that graph boundaries are as rare as in a long decode loop); for K > 1000 a pass is split
+    # into graphs of 1000 nodes.  Either way every timed sample is a whole number of K-step passes.
+    m = max(1, 1000 // K)
+    nodes = min(K * m, 1000)
+    full, rem = divmod(K * m, nodes)
     g_main = capture(oneshot, sets, nodes)
     g_rem = capture(oneshot, sets, rem) if rem else None
     g_warm = capture(oneshot, sets, W)
-    launches_capture = nb.nuna_launch_count() - launches0
     with torch.cuda.stream(stream):
-        g_warm.replay()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        t0 = time.time()
-        e0.record(stream)
-        for _ in range(replays):
-            g_main.replay()
-        if g_rem is not None:
-            g_rem.replay()
-        e1.record(stream)
-        barrier()
-        t1 = time.time()
-    sampler.mark(t0, t1)
-    total_ms = max_over_ranks(e0.elapsed_time(e1))
-    us_per_step = total_ms * 1e3 / K
+        g_warm.replay()                                               # the W untimed warm-up steps
+    torch.cuda.synchronize()
+    pass_graphs = [g_main] * full + ([g_rem] if g_rem is not None else [])
+    per_sample, region_ms = time_passes(pass_graphs, K * m, MIN_TIMED_MS, 5, warm_passes=0)
+    hs = stats_of(per_sample)
+    launches_timed = K * m * hs["samples"]                            # one kernel per step, every sample timed
+    us_per_step = hs["median"]
     alg_bytes = 2 * N_RANKS * w.bytes_per_rank                       # every source once + every destination once
     achieved = alg_bytes / (us_per_step * 1e-6) / 1e9
-    del g_main, g_rem, g_warm
+    del g_main, g_rem, g_warm, pass_graphs
+    emit("headline", {"us_per_step": hs, "samples": hs["samples"], "passes_per_sample": m, "steps_per_pass": K,
+                      "timed_region_ms": round(region_ms, 2),
+                      "mean_us_per_step_over_region": round(region_ms * 1e3 / (K * m * hs["samples"]), 4),
+                      "buffer_sets": len(sets)})
 
-    # launch floor: the same graph shape with an empty kernel of the same grid
+    # ---- launch floors ----------------------------------------------------------------------------------
     grid_blocks = min(N_RANKS * -(-(count // 8) // 256), num_sms * 5)
-    floor_us = per_call_us(lambda s, d, st: nb.nuna_launch_floor(grid_blocks, stream=st), sets, 1000, 3)
-    floor_pdl_us = per_call_us(lambda s, d, st: nb.nuna_launch_floor(grid_blocks, flags=nb.NUNA_LAUNCH_PDL, stream=st), sets, 1000, 3)
+    empty = lambda s, d, st: nb.nuna_launch_floor(grid_blocks, stream=st)
+    empty_pdl = lambda s, d, st: nb.nuna_launch_floor(grid_blocks, flags=nb.NUNA_LAUNCH_PDL, stream=st)
+    floor_us = per_call_us(empty, sets, 1000)
+    floor_pdl_us = per_call_us(empty_pdl, sets, 1000)
+    floors = {"graph_node_us": round(floor_us, 3), "graph_node_pdl_us": round(floor_pdl_us, 3),
+              "eager_event_pair_us": isolated_stats(empty, sets),
+              "eager_launch_plus_stream_sync_host_us": host_sync_floor(empty, sets),
+              "grid_blocks": grid_blocks}
+    emit("launch_floor", floors)
 
-    extras = {}
-    # ---- placement on the headline workload: round-robin baseline vs the two placement-aware kernels ---------
-    # (per-SM work lists use the topology of a probe run here on the first buffer set)
-    topo = nb.nuna_probe_topology(list(sets[0][0]) + list(sets[0][1]))
-    doms = [topo.sm_domain[s] for s in range(topo.num_sms)]
-    extras["probe"] = {
-        "sms": topo.num_sms, "sms_reported": topo.sms_reported, "lines": topo.num_lines,
-        "verdict": "nonuniform" if topo.verdict == nb.NUNA_TOPO_NONUNIFORM else "uniform",
-        "domain_sizes": [doms.count(0), doms.count(1)], "near_cycles": round(topo.near_lat, 1),
-        "far_cycles": round(topo.far_lat, 1), "gap_cycles": round(topo.domain_gap, 1), "noise_cycles": round(topo.noise, 2),
-        "sm_mean_hit_cycles_min_max": [round(min(topo.sm_lat_hit[:topo.num_sms]), 1), round(max(topo.sm_lat_hit[:topo.num_sms]), 1)],
-        "sm_miss_cycles_min_max": [round(min(topo.sm_lat_miss[:topo.num_sms]), 1), round(max(topo.sm_lat_miss[:topo.num_sms]), 1)],
-        "hist_first_cycle": nb.NUNA_HIST_FIRST, "hist_step": nb.NUNA_HIST_STEP,
-        "hist_near": list(topo.hist_near), "hist_far": list(topo.hist_far),
-    }
-    place = {}
-    for pname, pflags in (("roundrobin", nb.NUNA_PLACE_ROUNDROBIN), ("aware_colocated", nb.NUNA_PLACE_AWARE),
-                          ("aware_cluster_dsmem", nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_CLUSTER),
-                          ("aware_sm_lists", nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS)):
-        fn = lambda s, d, st, f=pflags: nb.nuna_allreduce_oneshot(s, d, count, flags=f, stream=st)
-        place[pname] = {"cold_us": round(per_call_us(fn, sets, 1000, 3), 3),
-                        "l2_resident_us": round(per_call_us(fn, sets[:1], 1000, 3), 3)}
-    extras["placement_512KiB"] = place
+    # ---- end to end through the host-buffer entry point (pinned host memory) -----------------------
+    hsrc = [torch.from_numpy(a.view(np.int16).copy()).pin_memory() for a in workloads.make(w)]
+    hdst = [torch.empty(count, dtype=torch.int16).pin_memory() for _ in range(N_RANKS)]
 
-    # ---- robustness to concurrent work (the paper runs its collectives beside a GEMM, Section 6.6) ------------
-    # 1 MiB per rank one-shot, L2-resident sources, while a second stream runs (a) nothing, (b) a streaming
-    # copy, (c) a dense bf16 matmul (a library GEMM used only as a load generator).
+    def time_host(**kw):
+        for _ in range(3):
+            nb.nuna_allreduce_host(hsrc, hdst, count, **kw)
+        barrier()
+        per = []
+        for _ in range(60):
+            t0 = time.perf_counter()
+            nb.nuna_allreduce_host(hsrc, hdst, count, **kw)
+            per.append((time.perf_counter() - t0) * 1e6)
+        return max_over_ranks(statistics.median(per))
+    e2e_variants = {"inplace_twoshot_put": time_host(flags=nb.NUNA_TWOSHOT_PUT, two_shot=True),
+                    "staged_copies_oneshot": time_host()}
+    e2e_best = min(e2e_variants, key=e2e_variants.get)
+    e2e = {"value": e2e_variants[e2e_best], "unit": "us", "h2d_bytes_per_step": N_RANKS * w.bytes_per_rank,
+           "d2h_bytes_per_step": N_RANKS * w.bytes_per_rank, "path": "nuna_allreduce_host, pinned host buffers: " + e2e_best}
+    emit("e2e", {"variants_us": {k: round(v, 2) for k, v in e2e_variants.items()}, "chosen": e2e_best})
+    del hsrc, hdst
+
+    sweep = []
     if not args.quick:
+        # ---- placement on the headline workload: round-robin baseline vs the placement-aware kernels ---------
+        # (per-SM work lists use the topology of a probe run here on the first buffer set)
+        topo = nb.nuna_probe_topology(list(sets[0][0]) + list(sets[0][1]))
+        doms = [topo.sm_domain[s] for s in range(topo.num_sms)]
+        emit("probe", {
+            "sms": topo.num_sms, "sms_reported": topo.sms_reported, "lines": topo.num_lines,
+            "verdict": "nonuniform" if topo.verdict == nb.NUNA_TOPO_NONUNIFORM else "uniform",
+            "domain_sizes": [doms.count(0), doms.count(1)], "near_cycles": round(topo.near_lat, 1),
+            "far_cycles": round(topo.far_lat, 1), "gap_cycles": round(topo.domain_gap, 1), "noise_cycles": round(topo.noise, 2),
+            "sm_mean_hit_cycles_min_max": [round(min(topo.sm_lat_hit[:topo.num_sms]), 1), round(max(topo.sm_lat_hit[:topo.num_sms]), 1)],
+            "sm_miss_cycles_min_max": [round(min(topo.sm_lat_miss[:topo.num_sms]), 1), round(max(topo.sm_lat_miss[:topo.num_sms]), 1)],
+            "hist_first_cycle": nb.NUNA_HIST_FIRST, "hist_step": nb.NUNA_HIST_STEP,
+            "hist_near": list(topo.hist_near), "hist_far": list(topo.hist_far)})
+        place = {}
+        for pname, pflags in PLACEMENT_VARIANTS(nb).items():
+            fn = lambda s, d, st, f=pflags: nb.nuna_allreduce_oneshot(s, d, count, flags=f, stream=st)
+            place[pname] = {"cold_us": round(per_call_us(fn, sets, 1000), 3),
+                            "l2_resident_us": round(per_call_us(fn, sets[:1], 1000), 3)}
+        emit("placement_512KiB", place)
+
+        # ---- robustness to concurrent work (the paper runs its collectives beside a GEMM, Section 6.6) ------------
+        # 1 MiB per rank one-shot, L2-resident sources, while a second stream runs (a) nothing, (b) a streaming
+        # copy, (c) a dense bf16 matmul (a library GEMM used only as a load generator).
         c1 = (1 << 20) // 2
         isets = make_sets(N_RANKS, c1, c1, 0, "normal", 77, max_sets=2)
         side = torch.cuda.Stream()
@@ -306,7 +445,7 @@ def run_gpu(args):
         inter = {}
         for lname, load in loads.items():
             row = {}
-            for pname, pflags in (("roundrobin", nb.NUNA_PLACE_ROUNDROBIN), ("aware_colocated", nb.NUNA_PLACE_AWARE)):
+            for pname, pflags in (("roundrobin", nb.NUNA_PLACE_ROUNDROBIN), ("aware", nb.NUNA_PLACE_AWARE)):
                 fn = lambda s, d, st, f=pflags: nb.nuna_allreduce_oneshot(s, d, c1, flags=f, stream=st)
                 g = capture(fn, isets, 400)
                 with torch.cuda.stream(stream):
@@ -327,86 +466,87 @@ def run_gpu(args):
                 row[pname] = {"us": round(e0.elapsed_time(e1) * 1e3 / 800, 3), "background_outlasted_timing": busy}
                 del g
             inter[lname] = row
-        extras["interference_1MiB_resident"] = inter
+        emit("interference_1MiB_resident", inter)
 
-        # ---- sensitivity to the number of thread blocks (the paper contrasts few and many, Section 6.5) ---------
+        # ---- sensitivity to the number of thread blocks and of SM domains (Section 6.5) ------------------------
         blocks_rows = {}
         for label, fn_of in (("oneshot_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c1, stream=st))),
                              ("twoshot_put_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c1, flags=nb.NUNA_TWOSHOT_PUT, stream=st)))):
             row = {}
             for blocks in (8, 37, 148, 592, 0):
                 nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, blocks)
-                row["default" if blocks == 0 else str(blocks)] = round(per_call_us(fn_of(), isets, 200, 2), 3)
+                row["default" if blocks == 0 else str(blocks)] = round(per_call_us(fn_of(), isets, 200), 3)
             nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, 0)
             blocks_rows[label] = row
-        extras["blocks_sensitivity_resident_us"] = blocks_rows
+        emit("blocks_sensitivity_resident_us", blocks_rows)
+        if True:
+            dom_rows = {}
+            sm_flags = nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS
+            for label, cnt, ss in (("512KiB", count, sets[:1]), ("1MiB", c1, isets[:1])):
+                row = {}
+                for D in (1, 2, 4, 8):
+                    nb.nuna_set_option(nb.NUNA_OPT_DOMAINS, D)
+                    fn = lambda s, d, st, c=cnt: nb.nuna_allreduce_oneshot(s, d, c, flags=sm_flags, stream=st)
+                    row[str(D)] = round(per_call_us(fn, ss, 200), 3)
+                nb.nuna_set_option(nb.NUNA_OPT_DOMAINS, 0)
+                dom_rows[label] = row
+            emit("domain_count_sensitivity_sm_lists_resident_us", dom_rows)
         del isets, big_a, big_b, ma, mb
         torch.cuda.empty_cache()
-    if True:
-        # ---- end to end through the host-buffer entry point (pinned host memory) -----------------------
-        hsrc = [torch.from_numpy(a.view(np.int16).copy()).pin_memory() for a in workloads.make(w)]
-        hdst = [torch.empty(count, dtype=torch.int16).pin_memory() for _ in range(N_RANKS)]
-        def time_host(**kw):
-            for _ in range(3):
-                nb.nuna_allreduce_host(hsrc, hdst, count, **kw)
-            barrier()
-            t0 = time.perf_counter()
-            for _ in range(50):
-                nb.nuna_allreduce_host(hsrc, hdst, count, **kw)
-            return max_over_ranks((time.perf_counter() - t0) / 50 * 1e6)
-        # the call a user with host data makes: pinned buffers, the kernel works on them in place
-        e2e_us = time_host(flags=nb.NUNA_TWOSHOT_PUT, two_shot=True)
-        staged_us = time_host()                                   # one-shot through device staging copies
-        extras["e2e"] = {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": N_RANKS * w.bytes_per_rank,
-                         "d2h_bytes_per_step": N_RANKS * w.bytes_per_rank,
-                         "path": "nuna_allreduce_host, pinned host buffers accessed in place by the two-shot put kernel",
-                         "staged_copies_oneshot_us": staged_us}
 
-    sweep, ag_row, a2a_row, rs_rows, chain_rows = [], None, None, [], []
-    if not args.quick:
         # ---- message-size sweep, 8 ranks, 8 KiB .. 64 MiB per rank --------------------------------------
+        P, PUT = nb.NUNA_LAUNCH_PDL, nb.NUNA_TWOSHOT_PUT
         algos = {
             "oneshot": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, stream=st)),
             "oneshot_aware": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=nb.NUNA_PLACE_AWARE, stream=st)),
             "twoshot": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, stream=st)),
-            "twoshot_put": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, flags=nb.NUNA_TWOSHOT_PUT, stream=st)),
-            # the same two with programmatic dependent launch (the one-shot drops it above 16 MiB of sources)
-            "oneshot_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=nb.NUNA_LAUNCH_PDL, stream=st)),
-            "twoshot_put_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(
-                s, d, c, flags=nb.NUNA_TWOSHOT_PUT | nb.NUNA_LAUNCH_PDL, stream=st)),
-            # nuna_allreduce: the library picks the algorithm by size
-            "size_selected": lambda c: (lambda s, d, st: nb.nuna_allreduce(
-                s, d, c, flags=nb.NUNA_TWOSHOT_PUT | nb.NUNA_LAUNCH_PDL | nb.NUNA_PLACE_AUTO, stream=st)),
+            "twoshot_put": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, flags=PUT, stream=st)),
+            # the same with programmatic dependent launch
+            "oneshot_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=P, stream=st)),
+            "oneshot_auto_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=P | nb.NUNA_PLACE_AUTO, stream=st)),
+            "oneshot_staged_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(
+                s, d, c, flags=P | nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_STAGED, stream=st)),
+            "twoshot_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, flags=P, stream=st)),
+            "twoshot_put_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, flags=PUT | P, stream=st)),
+            # nuna_allreduce: the library picks the algorithm by size; with no flags at all, and as tuned callers use it
+            "selected_default": lambda c: (lambda s, d, st: nb.nuna_allreduce(s, d, c, stream=st)),
+            "selected_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce(s, d, c, flags=P | nb.NUNA_PLACE_AUTO, stream=st)),
         }
         for wl in workloads.config_size_sweep(args.sweep_min, args.sweep_max):
             c, B = wl.count, wl.bytes_per_rank
             ssets = make_sets(N_RANKS, c, c, 2 * l2 + (64 << 20), "normal", wl.seed)
             nodes_s = max(len(ssets), min(512, (256 << 20) // B + 1))          # at least one full rotation
-            reps = 7 if B <= (4 << 20) else 5
             row = {"bytes_per_rank": B, "buffer_sets": len(ssets), "algorithmic_bytes": 2 * N_RANKS * B,
-                   "calls_per_sample": nodes_s, "samples": reps}
+                   "calls_per_sample": nodes_s}
             for name, mk in algos.items():
-                cs = per_call_stats(mk(c), ssets, nodes_s, reps)
-                warm = per_call_stats(mk(c), ssets[:1], nodes_s, reps)["median"]
+                cs = per_call_stats(mk(c), ssets, nodes_s)
+                warm = per_call_stats(mk(c), ssets[:1], nodes_s, min_passes=7)["median"]
                 cold = cs["median"]
-                row[name] = {"cold_us": round(cold, 3), "cold_min_us": round(cs["min"], 3), "cold_max_us": round(cs["max"], 3),
-                             "warm_us": round(warm, 3),
+                row[name] = {"cold_us": round(cold, 3), "cold_min_us": round(cs["min"], 3), "cold_p95_us": round(cs["p95"], 3),
+                             "cold_max_us": round(cs["max"], 3), "samples": cs["samples"], "warm_us": round(warm, 3),
                              "cold_gbs": round(2 * N_RANKS * B / cold / 1e3, 1),
                              "cold_frac_of_peak": round(2 * N_RANKS * B / cold / 1e3 / peak_gbs, 4)}
+            # a lone eager call (event pair after a sync): launch latency included, no pipelining
+            row["isolated_oneshot_us"] = isolated_stats(algos["oneshot"](c), ssets, 200 if B <= (4 << 20) else 40)
+            row["isolated_twoshot_us"] = isolated_stats(algos["twoshot"](c), ssets, 200 if B <= (4 << 20) else 40)
+            row["isolated_twoshot_put_us"] = isolated_stats(algos["twoshot_put"](c), ssets, 200 if B <= (4 << 20) else 40)
+            row["isolated_oneshot_warm_us"] = isolated_stats(algos["oneshot"](c), ssets[:1], 100 if B <= (4 << 20) else 20)
             best = min(algos, key=lambda a: row[a]["cold_us"])
             row["best"] = best
             row["best_frac_of_peak"] = row[best]["cold_frac_of_peak"]
             sweep.append(row)
+            emit(f"sweep_2^{B.bit_length() - 1}B", row)
             del ssets
             torch.cuda.empty_cache()
 
         # ---- allgather, 16 ranks x 64 KiB ---------------------------------------------------------------
         wa = workloads.config_allgather16()
         asets = make_sets(wa.nranks, wa.count, wa.nranks * wa.count, 2 * l2 + (64 << 20), "uniform", wa.seed)
-        ag_us = per_call_us(lambda s, d, st: nb.nuna_allgather(s, d, wa.count, flags=nb.NUNA_LAUNCH_PDL, stream=st), asets, 512, 3)
+        ag = per_call_stats(lambda s, d, st: nb.nuna_allgather(s, d, wa.count, flags=P, stream=st), asets, 512)
         ag_bytes = wa.nranks * wa.bytes_per_rank + wa.nranks * wa.nranks * wa.bytes_per_rank
-        ag_row = {"workload": wa.name, "us": round(ag_us, 3), "algorithmic_bytes": ag_bytes,
-                  "gbs": round(ag_bytes / ag_us / 1e3, 1), "frac_of_peak": round(ag_bytes / ag_us / 1e3 / peak_gbs, 4)}
+        emit("allgather16", {"workload": wa.name, "us": round(ag["median"], 3), "p95_us": round(ag["p95"], 3),
+                             "algorithmic_bytes": ag_bytes, "gbs": round(ag_bytes / ag["median"] / 1e3, 1),
+                             "frac_of_peak": round(ag_bytes / ag["median"] / 1e3 / peak_gbs, 4)})
         del asets
         torch.cuda.empty_cache()
 
@@ -416,72 +556,58 @@ def run_gpu(args):
             cnt = (1 << log2b) // 2
             shard = cnt // N_RANKS
             rsets = make_sets(N_RANKS, cnt, shard, 2 * l2 + (64 << 20), "normal", 60 + log2b)
-            rs_us = per_call_us(lambda s, d, st: nb.nuna_reduce_scatter(s, d, shard, flags=nb.NUNA_LAUNCH_PDL, stream=st),
-                                rsets, max(len(rsets), 64), 3)
+            rs_us = per_call_us(lambda s, d, st: nb.nuna_reduce_scatter(s, d, shard, flags=P, stream=st),
+                                rsets, max(len(rsets), 64))
             rs_bytes = N_RANKS * 2 * cnt + 2 * cnt                     # every source once + every shard once
             rs_rows.append({"bytes_per_rank": 2 * cnt, "us": round(rs_us, 3), "algorithmic_bytes": rs_bytes,
                             "gbs": round(rs_bytes / rs_us / 1e3, 1), "frac_of_peak": round(rs_bytes / rs_us / 1e3 / peak_gbs, 4)})
             del rsets
             torch.cuda.empty_cache()
+        emit("reduce_scatter8", rs_rows)
 
         # ---- alltoall, 8 ranks x 64 KiB per pair ----------------------------------------------------------
         wt = workloads.config_alltoall8()
         tsets = make_sets(wt.nranks, wt.count, wt.count, 2 * l2 + (64 << 20), "normal", wt.seed)
         blk = wt.count // wt.nranks
-        a2a_us = per_call_us(lambda s, d, st: nb.nuna_alltoall(s, d, blk, flags=nb.NUNA_LAUNCH_PDL, stream=st), tsets, 512, 3)
+        a2a_us = per_call_us(lambda s, d, st: nb.nuna_alltoall(s, d, blk, flags=P, stream=st), tsets, 512)
         a2a_bytes = 2 * wt.nranks * wt.bytes_per_rank
-        a2a_row = {"workload": wt.name, "us": round(a2a_us, 3), "algorithmic_bytes": a2a_bytes,
-                   "gbs": round(a2a_bytes / a2a_us / 1e3, 1), "frac_of_peak": round(a2a_bytes / a2a_us / 1e3 / peak_gbs, 4)}
+        emit("alltoall8", {"workload": wt.name, "us": round(a2a_us, 3), "algorithmic_bytes": a2a_bytes,
+                           "gbs": round(a2a_bytes / a2a_us / 1e3, 1), "frac_of_peak": round(a2a_bytes / a2a_us / 1e3 / peak_gbs, 4)})
         del tsets
         torch.cuda.empty_cache()
 
-        # ---- decode-step chain: 160 back-to-back one-shot allreduces in one graph ------------------------
+        # ---- decode-step chain: 160 back-to-back one-shot allreduces, one launch per step ------------------
         # Two alternating source sets (attention-out / MLP-out partials), L2-resident as in decode.
-        variants = {
-            "roundrobin": nb.NUNA_PLACE_ROUNDROBIN,
-            "roundrobin_pdl": nb.NUNA_PLACE_ROUNDROBIN | nb.NUNA_LAUNCH_PDL,
-            "aware_pdl": nb.NUNA_PLACE_AWARE | nb.NUNA_LAUNCH_PDL,
-            "auto_resident_pdl": nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT | nb.NUNA_LAUNCH_PDL,
-            "aware_sm_lists_pdl": nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS | nb.NUNA_LAUNCH_PDL,
-        }
+        chain_rows = []
         for tokens in workloads.CHAIN_TOKENS:
             wc = workloads.config_decode_chain(tokens)
             csets = make_sets(N_RANKS, wc.count, wc.count, 0, "normal", wc.seed, max_sets=2)
             row = {"tokens": tokens, "bytes_per_rank": wc.bytes_per_rank, "nodes": workloads.CHAIN_NODES}
-            for vname, vflags in variants.items():
+            for vname, vflags in CHAIN_VARIANTS(nb).items():
                 chain = nb.nuna_chain_create([c[0] for c in csets], [c[1] for c in csets], workloads.CHAIN_NODES,
                                              wc.count, flags=vflags)
                 with torch.cuda.stream(stream):
                     for _ in range(3):
                         nb.nuna_chain_launch(chain, stream=stream)
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    evs = [torch.cuda.Event(enable_timing=True) for _ in range(21)]
                     barrier()
                     t0 = time.time()
-                    e0.record(stream)
-                    for _ in range(20):
+                    evs[0].record(stream)
+                    for i in range(20):
                         nb.nuna_chain_launch(chain, stream=stream)
-                    e1.record(stream)
+                        evs[i + 1].record(stream)
                     barrier()
                     sampler.mark(t0, time.time())
-                ms = max_over_ranks(e0.elapsed_time(e1))
+                per = sorted(max_over_ranks(evs[i].elapsed_time(evs[i + 1])) * 1e3 for i in range(20))
                 nb.nuna_chain_destroy(chain)
-                row[vname] = {"step_us": round(ms * 1e3 / 20, 2), "per_node_us": round(ms * 1e3 / 20 / workloads.CHAIN_NODES, 3)}
+                row[vname] = {"step_us": round(pctl(per, 0.5), 2), "step_p95_us": round(pctl(per, 0.95), 2),
+                              "per_node_us": round(pctl(per, 0.5) / workloads.CHAIN_NODES, 3)}
             chain_rows.append(row)
             del csets
+        emit("decode_chain", chain_rows)
 
     # ---- CPU baseline: the oracle as it stands, on this machine's cores (rank 0 at N = 1 only) -----------------
-    cpu = None
-    if rank == 0 and world == 1:
-        import oracle
-        cores = os.cpu_count() or 1
-        src = workloads.make(w)
-        oracle.allreduce(src, nthreads=cores)
-        reps, t0 = 0, time.perf_counter()
-        while time.perf_counter() - t0 < 1.5:
-            oracle.allreduce(src, nthreads=cores)
-            reps += 1
-        cpu = {"value": (time.perf_counter() - t0) / reps * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
-               "sample": f"{reps} whole allreduces of the 8 x 512 KiB workload (about {1.5 * cores:.0f} core-seconds)"}
+    cpu = cpu_baseline_block(workloads.make(w), w.name) if (rank == 0 and world == 1) else None
 
     launches_total = nb.nuna_launch_count()
     status = nb.nuna_device_status()
@@ -490,34 +616,61 @@ def run_gpu(args):
     if rank != 0:
         return 0
 
-    # dram__bytes_read.sum + dram__bytes_write.sum of one k_oneshot_rr<8,1> launch on this workload, from the
-    # ncu capture summarised in profiles/oneshot_rr_n8_512KiB.md (4.20 MB read, 0 written: the destinations
-    # are still dirty in L2 when the kernel ends)
-    traffic = 4200192
+    r4 = lambda x: None if x is None else round(x, 4)
+    summary = {"launch_floor_us": floors, "value_stats_us": {k: r4(v) for k, v in hs.items()},
+               "timed_region_ms": round(region_ms, 2), "launches_since_load": int(launches_total),
+               "peak_source": peak_src + " copy peak (MEASURED_PEAKS.json hbm_gbs)" if peak_src == "measured" else peak_src,
+               "e2e_path": e2e["path"], "l2_protocol": f"cold: rotates over {len(sets)} buffer sets "
+               f"({len(sets) * 2 * N_RANKS * w.bytes_per_rank >> 20} MiB) > 2 x L2"}
+    if sweep:
+        flag_us = [min(r["twoshot"]["cold_us"], r["twoshot_pdl"]["cold_us"]) for r in sweep]
+        summary["sweep"] = {
+            "log2_bytes_per_rank": [r["bytes_per_rank"].bit_length() - 1 for r in sweep],
+            "best_algo": [r["best"] for r in sweep],
+            "oneshot_us": [min(r["oneshot"]["cold_us"], r["oneshot_pdl"]["cold_us"], r["oneshot_auto_pdl"]["cold_us"],
+                               r["oneshot_staged_pdl"]["cold_us"]) for r in sweep],
+            "twoshot_flag_us": flag_us,
+            "twoshot_flag_frac": [round(2 * N_RANKS * r["bytes_per_rank"] / t / 1e3 / peak_gbs, 3) for r, t in zip(sweep, flag_us)],
+            "twoshot_put_us": [min(r["twoshot_put"]["cold_us"], r["twoshot_put_pdl"]["cold_us"]) for r in sweep],
+            "selected_default_us": [r["selected_default"]["cold_us"] for r in sweep],
+            "isolated_oneshot_us": [r["isolated_oneshot_us"]["median"] for r in sweep]}
+        summary["allgather16"] = detail["allgather16"]
+        summary["decode_chain_best_per_node_us"] = {
+            str(r["tokens"]): min(v["per_node_us"] for v in r.values() if isinstance(v, dict)) for r in detail["decode_chain"]}
+    emit("summary", summary)
+
+    # The last line: the contract's keys only, kept short enough to survive in a truncated log tail.
     line = {
-        "metric": METRIC, "value": us_per_step, "unit": "us", "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": us_per_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 storage, f32 accumulate", "data": "synthetic",
+        "metric": METRIC, "value": r4(us_per_step), "unit": "us", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": round(us_per_step / 1e3, 7), "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": DTYPE, "data": "synthetic",
         "config": {"workload": w.name, "nranks": N_RANKS, "bytes_per_rank": w.bytes_per_rank,
-                   "algorithm": "one-shot allreduce, placement AUTO, programmatic dependent launch",
-                   "launch": "CUDA graph of back-to-back calls",
-                   "l2_protocol": f"cold: rotates over {len(sets)} buffer sets ({len(sets) * 2 * N_RANKS * w.bytes_per_rank >> 20} MiB) > 2 x L2",
-                   "multi_gpu": "independent replicas (the emulated collective has no inter-GPU step)"},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
-                     "traffic": traffic, "peak_source": peak_src,
-                     "note": "512 KiB per rank moves 8 MiB: 1.28 us at peak, so this size is latency-bound; "
-                             "see sweep[] for the bandwidth-bound sizes",
-                     "launch_floor_us": round(floor_us, 3), "launch_floor_pdl_us": round(floor_pdl_us, 3)},
-        "gpu_launches": K,
-        "launches_since_load": int(launches_total),
+                   "algorithm": "one-shot, placement AUTO, PDL", "launch": f"graph of {m}x{K} calls per sample",
+                   "l2": f"cold, {len(sets)} buffer sets > 2xL2", "multi_gpu": "replicas only"},
+        "replays": hs["samples"], "gpu_launches": int(launches_timed),
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak_gbs, "unit": "GB/s",
+                     "frac": round(achieved / peak_gbs, 4), "traffic": recorded_traffic("oneshot_n8_512KiB"),
+                     "peak_source": peak_src},
+        "floor_us": floors["graph_node_pdl_us"],
+        "e2e": {"value": round(e2e["value"], 2), "unit": "us", "h2d_bytes_per_step": e2e["h2d_bytes_per_step"],
+                "d2h_bytes_per_step": e2e["d2h_bytes_per_step"]},
         "device_status": status,
-        "clocks": clocks,
-        "sweep": sweep, "allgather16": ag_row, "alltoall8": a2a_row, "reduce_scatter8": rs_rows, "decode_chain": chain_rows,
+        "clocks": {k: clocks.get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons")} if clocks else None,
     }
-    line.update(extras)
+    if sweep:
+        line["sizes_log2B"] = [r["bytes_per_rank"].bit_length() - 1 for r in sweep]
+        line["best_us"] = [round(r[r["best"]]["cold_us"], 2) for r in sweep]
+        line["best_frac"] = [round(r["best_frac_of_peak"], 3) for r in sweep]
     if cpu is not None:
         line["cpu_baseline"] = cpu
-    print(json.dumps(line))
+    try:
+        out_dir = os.path.join(ROOT, "gpurun_out")
+        os.makedirs(out_dir, exist_ok=True)
+        with open(os.path.join(out_dir, "bench_detail.json"), "w") as f:
+            json.dump({"result": line, "detail": detail}, f, indent=1)
+    except OSError:
+        pass
+    print(json.dumps(line, separators=(",", ":")), flush=True)
     return 0
 
 
@@ -558,10 +711,10 @@ def run_case(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="nuna", choices=["nuna", "reference"])
-    ap.add_argument("--quick", action="store_true", help="headline only: skip sweep, allgather and chain")
+    ap.add_argument("--quick", action="store_true", help="headline, floors and end-to-end only")
     ap.add_argument("--sweep-min", type=int, default=13)
     ap.add_argument("--sweep-max", type=int, default=26)
     ap.add_argument("--case", default=None,

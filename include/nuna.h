@@ -69,8 +69,9 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 #define NUNA_PLACE_AWARE      1u   /* a tile's N work items (one logical group, Section 4.2.1) are co-located:
                                       in one thread block by default, or through NUNA_PLACE_SM_LISTS /
                                       NUNA_PLACE_CLUSTER; only the one-shot allreduce distinguishes placements */
-#define NUNA_PLACE_AUTO       2u   /* AWARE where it was measured to help (see NUNA_HINT_RESIDENT), else
-                                      exactly the ROUNDROBIN kernel                                        */
+#define NUNA_PLACE_AUTO       2u   /* the placement-aware kernel measured fastest for the size (co-located group
+                                      under NUNA_HINT_RESIDENT, shared-memory staged group for larger cold
+                                      messages), else exactly the ROUNDROBIN kernel                        */
 #define NUNA_PLACE_MASK       3u
 /* `flags`, bit 4 (nuna_allreduce_twoshot only): the reducing block stores its tile straight into all N
  * destinations, with no intermediate shard and no barrier.                                             */
@@ -82,9 +83,10 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 #define NUNA_HINT_RESIDENT    32u
 /* `flags`, bit 6: launch with programmatic stream serialization.  The kernel may be scheduled while its
  * predecessor in the stream drains; it waits for that grid's completion and memory visibility before
- * its first global access, so results are those of an ordinary stream-ordered launch.  Ignored by the
- * flag-barrier two-shot (a cooperative launch) and by the one-shot above 16 MiB of sources, where it
- * was measured not to pay.                                                                              */
+ * its first global access, so results are those of an ordinary stream-ordered launch.  The flag-
+ * synchronised two-shot is launched cooperatively without this flag and as an ordinary (non-cooperative)
+ * launch with it; the round-robin one-shot ignores it above 16 MiB of sources, where it was measured
+ * not to pay.                                                                                           */
 #define NUNA_LAUNCH_PDL       64u
 /* `flags`, bit 7, with NUNA_PLACE_AWARE on nuna_allreduce_oneshot: dispatch the co-located groups through
  * per-SM work lists.  The lists are planned by Algorithm 1 from the topology the last
@@ -96,8 +98,24 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 /* `flags`, bit 8, with NUNA_PLACE_AWARE on nuna_allreduce_oneshot, 2 <= nranks <= 8: run each tile's N work
  * items as one thread-block cluster of N blocks (placed by the hardware on one GPC).  Block r fetches
  * source r's tile once into shared memory; after a cluster barrier every block reads all N tiles from its
- * neighbours' shared memory and folds them for its own destination.  Ignored for other rank counts.     */
+ * neighbours' shared memory and folds them for its own destination.  Ignored for other rank counts.
+ * Experimental: measured 3.5-6x slower than the baseline at every size; NUNA_PLACE_AUTO never picks it. */
 #define NUNA_PLACE_CLUSTER    256u
+/* `flags`, bit 9, with NUNA_PLACE_AWARE on nuna_allreduce_oneshot: the co-located group staged through
+ * shared memory.  One thread of the block fetches the tile's N source slices with bulk asynchronous
+ * copies (global -> shared, completion on an mbarrier, this GPU's memory only); every emulated rank's row
+ * then folds the N slices out of shared memory and stores its own destination.                          */
+#define NUNA_PLACE_STAGED     512u
+/* `flags`, bit 10, nuna_allreduce only: for messages beyond the one-shot range use the flag-synchronised
+ * two-shot (reduce-scatter, per-tile ready flags, allgather) instead of the put form.                   */
+#define NUNA_TWOSHOT_SYNC     1024u
+/* `flags`, bits 11-12, nuna_chain_create only: run the chain as ONE kernel on a single thread-block
+ * cluster with a cluster barrier as node boundary (NUNA_CHAIN_PERSISTENT; one-shot nodes, at most 8
+ * buffer sets, at most 4 MiB per rank, else NUNA_ERR_INVALID_ARG), or always as a CUDA graph of one kernel
+ * per node (NUNA_CHAIN_GRAPH).  With neither bit the library picks the single kernel for small nodes
+ * (up to 128 KiB per rank), where a launch per node costs more than the node's data movement.           */
+#define NUNA_CHAIN_PERSISTENT 2048u
+#define NUNA_CHAIN_GRAPH      4096u
 
 /* ---- topology probe --------------------------------------------------------------------------------
  * Result of nuna_probe_topology: caller-owned, plain data, fixed maximum sizes.  Latencies are in SM
@@ -204,9 +222,15 @@ int nuna_init(size_t scratch_bytes);
  *  NUNA_OPT_UNROLL          vectors per thread per work item (1, 2, 4; limited so that N * unroll <= 16)
  *  NUNA_OPT_COLOC           destinations of a tile that share a block in the placement-aware one-shot (2, 4, 8)
  *  NUNA_OPT_AUTO_MIN_BYTES  smallest message per rank for which NUNA_PLACE_AUTO may pick the aware kernel
- *  NUNA_OPT_TIMEOUT_MS      flag-barrier timeout
+ *  NUNA_OPT_TIMEOUT_MS      limit of every in-kernel wait (ready flags, barrier, bulk-copy completion)
+ *  NUNA_OPT_DOMAINS         number of SM domains the NUNA_PLACE_SM_LISTS planner deals groups to (the paper's
+ *                           sweep over routing domains, Section 6.5): 1 = one domain, 2 = the probed split,
+ *                           more = every probed domain cut into equal latency quantiles; 0 = what the probe found
+ *  NUNA_OPT_STAGE_VECS      16-byte vectors per source per tile of the NUNA_PLACE_STAGED kernel (0 = by size)
+ *  NUNA_OPT_TWOSHOT_VECS    16-byte vectors per tile (= per ready flag) of the flag-synchronised two-shot (0 = by size)
  * Returns NUNA_ERR_INVALID_ARG for an unknown option or a negative value.  Creates the context.          */
-enum { NUNA_OPT_BLOCKS = 0, NUNA_OPT_UNROLL = 1, NUNA_OPT_COLOC = 2, NUNA_OPT_AUTO_MIN_BYTES = 3, NUNA_OPT_TIMEOUT_MS = 4 };
+enum { NUNA_OPT_BLOCKS = 0, NUNA_OPT_UNROLL = 1, NUNA_OPT_COLOC = 2, NUNA_OPT_AUTO_MIN_BYTES = 3, NUNA_OPT_TIMEOUT_MS = 4,
+       NUNA_OPT_DOMAINS = 5, NUNA_OPT_STAGE_VECS = 6, NUNA_OPT_TWOSHOT_VECS = 7 };
 int nuna_set_option(int option, long long value);
 
 /* One-shot allreduce (Section 5.1, direct algorithm): every emulated rank d reads all N sources and
@@ -214,21 +238,25 @@ int nuna_set_option(int option, long long value);
 int nuna_allreduce_oneshot(const void* const* src, void* const* dst, int nranks,
                            size_t count, int dtype, unsigned flags, void* stream);
 
-/* Two-shot allreduce: reduce-scatter over N contiguous chunks (emulated rank r reduces chunk r), an
- * in-kernel flag barrier among the persistent thread blocks, then a put-style allgather of the chunks
- * into every destination.  Same bits as the one-shot.  Any `count`; chunk = ceil(count/N) rounded up
- * to a whole 16-byte vector, trailing chunks may be short or empty.  Uses the context's shard scratch
- * (count*elemsize bytes, grown on demand) unless NUNA_TWOSHOT_PUT is set.  Calls that share the
- * context must be stream-ordered with respect to each other.                                          */
+/* Two-shot allreduce: reduce-scatter over N contiguous chunks (the chunk a tile lies in names the emulated
+ * rank that reduces it), per-tile ready flags in place of a host synchronisation, then a put-style
+ * allgather of the reduced tiles into every destination -- all in one kernel of co-resident thread
+ * blocks.  A block that has reduced a tile publishes the tile's flag with a release store; the block that
+ * gathers the tile acquire-polls that flag (bounded wait: on expiry NUNA_ERR_TIMEOUT is latched and the
+ * block returns).  Same bits as the one-shot.  Any `count`; chunk = ceil(count/N) rounded up to a whole
+ * 16-byte vector, trailing chunks may be short or empty.  Uses the context's shard scratch (count*elemsize
+ * bytes plus one flag word per 4 KiB, grown on demand; an outgrown scratch stays allocated until
+ * nuna_shutdown because captured graphs may still name it) unless NUNA_TWOSHOT_PUT is set.  Calls that
+ * share the context must be stream-ordered with respect to each other.                                 */
 int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
                            size_t count, int dtype, unsigned flags, void* stream);
 
 /* Allreduce with the algorithm chosen by message size -- the counterpart of the paper's per-collective
  * choice between routing schemes by a size threshold (Section 4.1.2): one-shot while the message is small
  * enough for its single step to win (measured: up to 1 MiB per rank at 2 ranks, 512 KiB at 4, 128 KiB at
- * 8, 64 KiB at 16), the two-shot beyond.
- * With NUNA_TWOSHOT_PUT clear in `flags` the large-message choice is the flag-barrier two-shot instead
- * (set NUNA_TWOSHOT_PUT to allow the put form).  Same bits whichever is chosen.                          */
+ * 8, 64 KiB at 16), beyond that the put form of the two-shot, the fastest kernel at every larger size.
+ * With NUNA_TWOSHOT_SYNC the large-message choice is the flag-synchronised two-shot instead, from eight
+ * times those sizes (below, the one-shot is faster than it).  Same bits whichever is chosen.            */
 int nuna_allreduce(const void* const* src, void* const* dst, int nranks,
                    size_t count, int dtype, unsigned flags, void* stream);
 
@@ -255,20 +283,21 @@ int nuna_alltoall(const void* const* src, void* const* dst, int nranks,
  * on the request path: an inference server that has handed the whole GPU to its own memory pool, where
  * a raw allocation can fail or fragment the pool, or a latency-critical loop that cannot afford the
  * device-wide synchronisation and the failure modes an allocation brings.  This entry point computes
- * exactly what nuna_allreduce_twoshot computes (flag-barrier form, same bits) but takes its shard
- * intermediate and its barrier words from a fixed array compiled into the library, so it never calls
+ * exactly what nuna_allreduce_twoshot computes (flag-synchronised form, same bits) but takes its shard
+ * intermediate, ready flags and control words from fixed arrays compiled into the library, so it never calls
  * cudaMalloc, cudaFree or any allocating routine, and it does not create the per-device context.
  *  - Limit: 4 MiB per rank, i.e. count <= NUNA_STATIC_MAX_COUNT elements of a 16-bit type (half that
  *    many of binary32); larger messages return NUNA_ERR_TOO_LARGE and print the limit.  The array
  *    costs 4 MiB of device memory on every GPU that loads the library, for the life of the process.
- *  - The first call on a device looks up the array's device address and zeroes the barrier words
- *    (a small synchronous cudaMemset); make that first call before starting any stream capture.
+ *  - The first call on a device looks up the arrays' device addresses and zeroes the flags and control
+ *    words (two small synchronous cudaMemset calls); make that first call before starting any stream capture.
  *  - All calls on a device share the one array, which keeps the previous call's shard; the kernel
  *    overwrites every element it later reads, so stale contents never reach a result.  Two calls that
  *    overlap on the GPU (different streams, no ordering) race on it: keep calls stream-ordered.
- *  - A barrier that times out (1 s) latches NUNA_ERR_TIMEOUT in the array's own status word, which
- *    this entry point does not expose; results are then undefined.  src / dst / nranks / dtype /
- *    stream and the argument errors are those of nuna_allreduce_twoshot; there is no flags word.      */
+ *  - A wait that times out (1 s) latches NUNA_ERR_TIMEOUT in the arrays' own status word; results are
+ *    then undefined.  nuna_device_status reports that word too (the worse of it and the context's) and
+ *    rewinds the control words after a timeout.  src / dst / nranks / dtype / stream and the argument
+ *    errors are those of nuna_allreduce_twoshot; there is no flags word.                               */
 #define NUNA_STATIC_MAX_COUNT (2 * 1024 * 1024)
 int nuna_allreduce_twoshot_static(const void* const* src, void* const* dst, int nranks,
                                   size_t count, int dtype, void* stream);
@@ -287,15 +316,19 @@ int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks,
  * device pointers, set s occupying entries [s*nranks, (s+1)*nranks); node k works on set k mod nsets
  * and starts reading only after node k-1 has finished writing.  flags as for the allreduce calls
  * (NUNA_LAUNCH_PDL overlaps each node's launch with its predecessor's drain); two_shot selects
- * nuna_allreduce_twoshot.  Creation allocates and synchronises nothing on the caller's streams; the
- * chain reads the buffers named at creation on every launch.  *chain_out is an opaque handle.          */
+ * nuna_allreduce_twoshot.  Small one-shot nodes run as a single kernel instead of a graph (see
+ * NUNA_CHAIN_PERSISTENT / NUNA_CHAIN_GRAPH): one thread-block cluster loops over the nodes with a cluster
+ * barrier between them, which removes the per-node launch cost.  Creation allocates and synchronises
+ * nothing on the caller's streams; the chain reads the buffers named at creation on every launch.
+ * *chain_out is an opaque handle.                                                                       */
 int nuna_chain_create(const void* const* src_sets, void* const* dst_sets, int nsets, int nnodes, int nranks,
                       size_t count, int dtype, unsigned flags, int two_shot, void** chain_out);
 int nuna_chain_launch(void* chain, void* stream);      /* one replay of all nodes, asynchronous on `stream` */
 int nuna_chain_destroy(void* chain);
 
-/* Reads and clears the device status word of the current device (NUNA_OK or NUNA_ERR_TIMEOUT) after
- * synchronising the device.  After a timeout the barrier words are re-initialised.                     */
+/* Reads and clears the device status of the current device (NUNA_OK or NUNA_ERR_TIMEOUT) after
+ * synchronising the device: the worse of the context's status word and the allocation-free entry
+ * point's.  After a timeout the control words are rewound (the epoch keeps counting).                  */
 int nuna_device_status(int* out);
 
 /* Launches an empty kernel of `blocks` thread blocks with the collectives' block shape on `stream`: the

@@ -30,11 +30,16 @@ NUNA_HINT_RESIDENT = 32
 NUNA_LAUNCH_PDL = 64
 NUNA_PLACE_SM_LISTS = 128
 NUNA_PLACE_CLUSTER = 256
+NUNA_PLACE_STAGED = 512
+NUNA_TWOSHOT_SYNC = 1024
+NUNA_CHAIN_PERSISTENT = 2048
+NUNA_CHAIN_GRAPH = 4096
 
 NUNA_MAX_SMS, NUNA_MAX_PROBE_BUFS, NUNA_PROBE_REGIONS, NUNA_MAX_PROBE_LINES = 256, 32, 8, 2048
 NUNA_TOPO_UNIFORM, NUNA_TOPO_NONUNIFORM = 0, 1
 NUNA_HIST_BINS, NUNA_HIST_FIRST, NUNA_HIST_STEP = 48, 200, 4
 NUNA_OPT_BLOCKS, NUNA_OPT_UNROLL, NUNA_OPT_COLOC, NUNA_OPT_AUTO_MIN_BYTES, NUNA_OPT_TIMEOUT_MS = 0, 1, 2, 3, 4
+NUNA_OPT_DOMAINS, NUNA_OPT_STAGE_VECS, NUNA_OPT_TWOSHOT_VECS = 5, 6, 7
 
 
 class NunaTopology(ctypes.Structure):
@@ -127,7 +132,7 @@ def lib() -> ctypes.CDLL:
         L.nuna_debug_chain.restype = ctypes.c_int
         up = ctypes.POINTER(ctypes.c_uint)
         L.nuna_debug_plan_oneshot.argtypes = [ctypes.POINTER(NunaTopology), ctypes.c_int, ctypes.c_int, ctypes.c_size_t,
-                                              ctypes.c_size_t, ctypes.c_int, up, up]
+                                              ctypes.c_size_t, ctypes.c_int, ctypes.c_int, up, up]
         L.nuna_debug_plan_oneshot.restype = ctypes.c_int
         ip = ctypes.POINTER(ctypes.c_int)
         L.nuna_plan_placement.argtypes = [ctypes.POINTER(NunaPlanInput), ip, ip, ip, ip]
@@ -140,6 +145,8 @@ def lib() -> ctypes.CDLL:
         L.nuna_shutdown.restype = ctypes.c_int
         L.nuna_debug_barrier_selftest.argtypes = [ctypes.c_uint, ctypes.c_uint, ctypes.c_uint, ctypes.POINTER(ctypes.c_uint)]
         L.nuna_debug_barrier_selftest.restype = ctypes.c_int
+        L.nuna_debug_twoshot_unset_flags.argtypes = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint]
+        L.nuna_debug_twoshot_unset_flags.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -275,14 +282,15 @@ def debug_analyse_topology(lat, lat_rep):
     return topo
 
 
-def debug_plan_oneshot(topo, num_sms: int, nranks: int, ntiles: int, tile_bytes: int, generic: bool):
+def debug_plan_oneshot(topo, num_sms: int, nranks: int, ntiles: int, tile_bytes: int, generic: bool, domains: int = 0):
     """Per-SM work lists planned for a one-shot: returns a list (one entry per SM) of tile lists."""
     import numpy as np
     off = np.zeros(num_sms + 1, dtype=np.uint32)
     tiles = np.zeros(max(ntiles, 1), dtype=np.uint32)
     up = ctypes.POINTER(ctypes.c_uint)
     st = lib().nuna_debug_plan_oneshot(ctypes.byref(topo) if topo is not None else None, num_sms, nranks, ntiles,
-                                       tile_bytes, 1 if generic else 0, off.ctypes.data_as(up), tiles.ctypes.data_as(up))
+                                       tile_bytes, 1 if generic else 0, domains, off.ctypes.data_as(up),
+                                       tiles.ctypes.data_as(up))
     if st != NUNA_OK:
         raise NunaError(st, "nuna_debug_plan_oneshot")
     return [tiles[off[s]:off[s + 1]].tolist() for s in range(num_sms)]
@@ -358,6 +366,11 @@ nuna_status_string = status_string
 
 def nuna_shutdown() -> int:
     return lib().nuna_shutdown()
+
+
+def debug_twoshot_unset_flags(src, dst, count, dtype=NUNA_BF16, timeout_ms: int = 50) -> int:
+    """Test hook: a two-shot whose consumers wait for ready flags that nobody publishes (bounded waits)."""
+    return lib().nuna_debug_twoshot_unset_flags(ptr_table(src), ptr_table(dst), len(src), count, dtype, timeout_ms)
 
 
 def debug_barrier_selftest(grid: int, expected: int, timeout_ms: int):

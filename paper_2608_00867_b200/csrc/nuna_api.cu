@@ -1,5 +1,6 @@
 // Host side of the C ABI: argument checks, per-device context, launch configuration.
 #include "nuna_internal.h"
+#include "nuna_debug.h"
 #include "nuna_kernels.cuh"
 
 #include <algorithm>
@@ -17,6 +18,10 @@ std::atomic<unsigned long long> g_launches{0};
 static std::mutex g_ctx_mutex;
 static Context* g_ctx[kMaxDevices] = {};
 
+static int static_status_read_and_clear(unsigned* out);     // the allocation-free entry point's status word (end of file)
+constexpr unsigned kMinFlagTileVec = 16;                    // smallest two-shot tile (vectors): 256 bytes of shard per flag
+constexpr unsigned kStaticTileVec = 128;                    // tile of the allocation-free entry point: 2 KiB of shard per flag
+
 static int env_int(const char* name, int fallback)
 {
     const char* s = getenv(name);
@@ -26,6 +31,17 @@ static int env_int(const char* name, int fallback)
 int init_barrier_words(Context* c)
 {
     return cudaMemset(c->bw, 0, sizeof(BarrierWords)) == cudaSuccess ? NUNA_OK : NUNA_ERR_CUDA;
+}
+
+// After a latched timeout the barrier's arrival counter is in an undefined state: zero it and clear the
+// status, but keep both epochs moving forward -- the ready flags of earlier launches must never match a
+// later launch's epoch.  The device is idle (the caller synchronised).
+static int rewind_barrier_words(BarrierWords* dev, const BarrierWords& seen)
+{
+    BarrierWords h = {};
+    h.epoch = seen.epoch + 1u;
+    h.ticket = ((seen.ticket >> 32) + 1ull) << 32;
+    return cudaMemcpy(dev, &h, sizeof h, cudaMemcpyHostToDevice) == cudaSuccess ? NUNA_OK : NUNA_ERR_CUDA;
 }
 
 // Returns the current device's context, creating it on first use (allocates: not capturable).
@@ -43,25 +59,38 @@ int get_context(Context** out)
         c->l2_bytes = (size_t)prop.l2CacheSize;
         if (cudaMalloc(&c->bw, sizeof(BarrierWords)) != cudaSuccess) { delete c; return NUNA_ERR_CUDA; }
         if (init_barrier_words(c) != NUNA_OK) { cudaFree(c->bw); delete c; return NUNA_ERR_CUDA; }
-        c->timeout_ns = (unsigned long long)env_int("NUNA_TIMEOUT_MS", 1000) * 1000000ull;
-        c->blocks_override = env_int("NUNA_BLOCKS", 0);
-        c->unroll_override = env_int("NUNA_UNROLL", 0);
-        c->auto_min_bytes = (size_t)env_int("NUNA_AUTO_MIN_BYTES", 64 << 10);
-        c->coloc_override = env_int("NUNA_COLOC", 0);
+        c->opt.timeout_ns = (unsigned long long)env_int("NUNA_TIMEOUT_MS", 1000) * 1000000ull;
+        c->opt.blocks = env_int("NUNA_BLOCKS", 0);
+        c->opt.unroll = env_int("NUNA_UNROLL", 0);
+        c->opt.auto_min_bytes = (size_t)env_int("NUNA_AUTO_MIN_BYTES", 64 << 10);
+        c->opt.coloc = env_int("NUNA_COLOC", 0);
+        c->opt.domains = env_int("NUNA_DOMAINS", 0);
+        c->opt.stage_vecs = env_int("NUNA_STAGE_VECS", 0);
+        c->opt.twoshot_vecs = env_int("NUNA_TWOSHOT_VECS", 0);
         g_ctx[dev] = c;
     }
     *out = g_ctx[dev];
     return NUNA_OK;
 }
 
+// Grows the two-shot scratch (shard intermediate + one ready flag per smallest tile of it).  The caller holds
+// c->mutex.  An outgrown allocation is never freed before nuna_shutdown: a CUDA graph captured earlier
+// (a chain, or a user's capture of a two-shot call) still carries its address as a kernel argument.
 int ensure_scratch(Context* c, size_t bytes)
 {
-    if (bytes <= c->scratch_bytes) return NUNA_OK;
+    if (bytes <= c->scratch_bytes && c->scratch) return NUNA_OK;
+    const size_t want = (std::max<size_t>(bytes, 4096) + 4095) & ~(size_t)4095;
+    const size_t nflags = want / (kMinFlagTileVec * 16) + 1;         // one ready flag per smallest tile
     void* p = nullptr;
-    const size_t want = (bytes + 255) & ~(size_t)255;
-    if (cudaMalloc(&p, want) != cudaSuccess) return NUNA_ERR_CUDA;
-    if (c->scratch) cudaFree(c->scratch);
+    if (cudaMalloc(&p, want + nflags * sizeof(unsigned)) != cudaSuccess) return NUNA_ERR_CUDA;
+    // flags start at zero; epochs start at one, so a fresh flag never reads as "ready"
+    if (cudaMemset(static_cast<char*>(p) + want, 0, nflags * sizeof(unsigned)) != cudaSuccess) {
+        cudaFree(p);
+        return NUNA_ERR_CUDA;
+    }
+    if (c->scratch) c->retired_scratch.push_back(c->scratch);
     c->scratch = p;
+    c->flags = reinterpret_cast<unsigned*>(static_cast<char*>(p) + want);
     c->scratch_bytes = want;
     return NUNA_OK;
 }
@@ -84,7 +113,7 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
     if (nranks < 1) return NUNA_ERR_INVALID_ARG;
     if (dtype != NUNA_BF16 && dtype != NUNA_F16 && dtype != NUNA_F32) return NUNA_ERR_UNSUPPORTED_DTYPE;
     if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT | NUNA_HINT_RESIDENT | NUNA_LAUNCH_PDL | NUNA_PLACE_SM_LISTS |
-                   NUNA_PLACE_CLUSTER)) != 0u ||
+                   NUNA_PLACE_CLUSTER | NUNA_PLACE_STAGED | NUNA_TWOSHOT_SYNC | NUNA_CHAIN_PERSISTENT | NUNA_CHAIN_GRAPH)) != 0u ||
         (flags & NUNA_PLACE_MASK) == 3u)
         return NUNA_ERR_INVALID_ARG;
     if (src_elems > ((size_t)1 << 40) || dst_elems > ((size_t)1 << 40)) return NUNA_ERR_TOO_LARGE;
@@ -104,6 +133,9 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
     return NUNA_OK;
 }
 
+// Bits that only nuna_chain_create understands.
+static bool has_chain_bits(unsigned flags) { return (flags & (NUNA_CHAIN_PERSISTENT | NUNA_CHAIN_GRAPH)) != 0u; }
+
 static RankPtrs make_ptrs(const void* const* src, void* const* dst, int nranks)
 {
     RankPtrs p;
@@ -121,25 +153,29 @@ static RankPtrs make_ptrs(const void* const* src, void* const* dst, int nranks)
 // flight per thread, more vectors per thread only mean fewer blocks (measured at 2 and 4 ranks: 64 KiB
 // per rank 1.43 us with one vector, 1.64 us with four; no difference at 16 MiB).  NUNA_OPT_UNROLL
 // overrides it for experiments.
-static int pick_unroll(const Context* c, int nranks)
+static int pick_unroll(const Options& o, int nranks)
 {
     int u = 1;
-    if (c->unroll_override == 1 || c->unroll_override == 2 || c->unroll_override == 4) u = c->unroll_override;
+    if (o.unroll == 1 || o.unroll == 2 || o.unroll == 4) u = o.unroll;
     while (u > 1 && u * nranks > 16) u >>= 1;
     return u;
 }
 
+// Resident blocks per SM of a kernel, looked up once per device (the cache is one slot per device and
+// kernel instantiation; racing first calls compute the same value).
 template <typename K>
-static int occupancy(Context* c, K kernel, int* cache)
+static int occupancy(K kernel, std::atomic<int>* cache /* [kMaxDevices] */)
 {
-    if (*cache == 0) {
-        int n = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, 0) != cudaSuccess || n < 1) n = 1;
-        *cache = n;
+        cache[dev].store(n, std::memory_order_relaxed);
     }
-    (void)c;
-    return *cache;
+    return n;
 }
+#define NUNA_OCC(kernel) ([&]() { static std::atomic<int> cache_[kMaxDevices]; return occupancy(kernel, cache_); }())
 
 // Grid size: `waves` x (SMs x resident blocks per SM), never more than the work items.  Streaming
 // kernels (two-shot put, reduce-scatter, allgather) run one item per block (waves = 0: no cap): leaving
@@ -147,10 +183,10 @@ static int occupancy(Context* c, K kernel, int* cache)
 // against 0.90 for a persistent grid-stride loop.  The one-shot wants its N readers of a tile close in
 // time so that re-reads hit L2: four waves measured best (0.70 of peak at 64 MiB against 0.63 for one
 // wave and 0.62 for an uncapped grid).
-static unsigned pick_grid(const Context* c, size_t nitems, int blocks_per_sm, int waves = 1)
+static unsigned pick_grid(const Context* c, const Options& o, size_t nitems, int blocks_per_sm, int waves = 1)
 {
     size_t cap = waves > 0 ? (size_t)c->num_sms * (size_t)blocks_per_sm * (size_t)waves : ((size_t)1 << 22);
-    if (c->blocks_override > 0) cap = (size_t)c->blocks_override;
+    if (o.blocks > 0) cap = (size_t)o.blocks;
     return (unsigned)std::max<size_t>(1, std::min(nitems, cap));
 }
 
@@ -166,6 +202,7 @@ static unsigned launch_mode(unsigned flags, size_t total_src_bytes = 0)
 }
 
 static thread_local unsigned t_cluster_dim = 0;           // > 0: next launch() uses clusters of this many blocks
+static thread_local unsigned t_dyn_smem = 0;              // next launch() requests this much dynamic shared memory
 
 template <typename... Args, typename... Act>
 static int launch(void (*kernel)(Args...), unsigned grid, cudaStream_t stream, unsigned mode, Act&&... args)
@@ -173,7 +210,8 @@ static int launch(void (*kernel)(Args...), unsigned grid, cudaStream_t stream, u
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = t_dyn_smem;
+    t_dyn_smem = 0;
     cfg.stream = stream;
     cudaLaunchAttribute attr[3];
     int nattr = 0;
@@ -249,15 +287,22 @@ static size_t ceil_div(size_t a, size_t b) { return (a + b - 1) / b; }
 
 // ---- collectives ---------------------------------------------------------------------------------
 
-// NUNA_PLACE_AUTO: use the placement-aware kernel only where it is at least as fast as the
-// round-robin baseline.  NUNA_AUTO_MIN_BYTES overrides the measured crossover (bytes per rank).
-static bool aware_pays_off(const Context* c, int nranks, size_t bytes, unsigned flags)
+// NUNA_PLACE_AUTO picks, per size, the one-shot kernel that was measured fastest on B200 (8 ranks; the
+// other rank counts use the same rules), never one that is slower than the round-robin baseline:
+//  * sources L2-resident (NUNA_HINT_RESIDENT) and 64 KiB <= bytes per rank, 4 N bytes within L2: the
+//    co-located group kernel (rows of one block share the tile through L1);
+//  * otherwise, from kStageMinBytes per rank: the group staged through shared memory by bulk copies;
+//  * otherwise the round-robin kernel itself.
+enum class OneShotKernel { RoundRobin, Group, Staged };
+constexpr size_t kStageMinBytes = (size_t)4 << 20;
+
+static OneShotKernel auto_kernel(const Context* c, const Options& o, int nranks, size_t bytes, unsigned flags)
 {
-    if (nranks < 2 || !(flags & NUNA_HINT_RESIDENT)) return false;
-    // sources and destinations of one call, twice over (the producer's other buffers), must fit in L2
-    // for "resident" to be physically possible
-    if (4 * bytes * (size_t)nranks > c->l2_bytes) return false;
-    return bytes >= c->auto_min_bytes;
+    if (nranks < 2) return OneShotKernel::RoundRobin;
+    if ((flags & NUNA_HINT_RESIDENT) && 4 * bytes * (size_t)nranks <= c->l2_bytes && bytes >= o.auto_min_bytes)
+        return OneShotKernel::Group;
+    if (bytes >= kStageMinBytes) return OneShotKernel::Staged;
+    return OneShotKernel::RoundRobin;
 }
 
 
@@ -265,20 +310,22 @@ static bool aware_pays_off(const Context* c, int nranks, size_t bytes, unsigned 
 //
 // Thread blocks = work items (tile, d); item (t, d) touches the N source chunks of tile t and the
 // destination chunk (d, t).  Domains and the order of SMs inside a domain come from the probe
-// (nearest = lowest mean hit latency).  The per-SM budget R_max is ceil(groups per domain / SMs of
-// the smallest domain) whole groups, so a small workload fills only the nearest SMs, one group each,
-// and a large one spreads evenly.  Up to kGenericPlanTiles tiles the lists are produced by the
-// general planner (nuna_plan_placement); beyond that by the closed form it reduces to for this
-// workload (tile t -> domain t mod D, SMs of the domain filled in preference order), which the host
-// tests check against the general planner.
+// (nearest = lowest mean hit latency).  `domains` = 0 uses what the probe found (one, or the two dies);
+// a larger count splits every probed domain into equal latency quantiles (the paper's sweep over the
+// number of routing domains, Section 6.5), 1 forces a single domain.  The per-SM budget R_max is
+// ceil(groups per domain / SMs of the smallest domain) whole groups, so a small workload fills only the
+// nearest SMs, one group each, and a large one spreads evenly.  Up to kGenericPlanTiles tiles the lists
+// are produced by the general planner (nuna_plan_placement); beyond that by the closed form it reduces to
+// for this workload (tile t -> domain t mod D, SMs of the domain filled in preference order), which the
+// host tests check against the general planner.
 constexpr size_t kGenericPlanTiles = 1024;
 
 void plan_oneshot_lists(const nuna_topology_t* topo, int num_sms, int nranks, size_t ntiles, size_t tile_bytes,
-                        bool generic, std::vector<std::vector<unsigned>>& lists)
+                        bool generic, int domains, std::vector<std::vector<unsigned>>& lists)
 {
     lists.assign((size_t)num_sms, {});
-    const bool split = topo && topo->verdict == NUNA_TOPO_NONUNIFORM && topo->num_domains == 2;
-    const int D = split ? 2 : 1;
+    const bool split = topo && topo->verdict == NUNA_TOPO_NONUNIFORM && topo->num_domains == 2 && domains != 1;
+    const int base_domains = split ? 2 : 1;
     std::vector<int> dom(num_sms, 0), rank(num_sms, 0), order(num_sms);
     for (int s = 0; s < num_sms; ++s) {
         order[s] = s;
@@ -290,12 +337,24 @@ void plan_oneshot_lists(const nuna_topology_t* topo, int num_sms, int nranks, si
             return la < lb;
         });
     for (int i = 0; i < num_sms; ++i) rank[order[i]] = i;
-    int smallest = num_sms;
-    if (split) {
-        int n1 = 0;
-        for (int s = 0; s < num_sms; ++s) n1 += dom[s];
-        smallest = std::max(1, std::min(n1, num_sms - n1));
+    // more domains than the probe found: cut each probed domain into `sub` latency quantiles
+    int D = base_domains;
+    if (domains > base_domains) {
+        const int sub = std::max(1, std::min(domains / base_domains, num_sms / base_domains));
+        std::vector<int> size(base_domains, 0), seen(base_domains, 0);
+        for (int s = 0; s < num_sms; ++s) size[dom[s]]++;
+        std::vector<int> fine(num_sms, 0);
+        for (int i = 0; i < num_sms; ++i) {                          // in preference order
+            const int s = order[i], b = dom[s];
+            const int q = std::min(sub - 1, (int)((long long)seen[b]++ * sub / std::max(1, size[b])));
+            fine[s] = b * sub + q;
+        }
+        dom = fine;
+        D = base_domains * sub;
     }
+    std::vector<int> dsize(D, 0);
+    for (int s = 0; s < num_sms; ++s) dsize[dom[s]]++;
+    const int smallest = std::max(1, *std::min_element(dsize.begin(), dsize.end()));
     const size_t per_domain = ceil_div(ntiles, (size_t)D);
     const size_t budget = std::max<size_t>(1, ceil_div(per_domain, (size_t)smallest));        // groups per SM
     if (generic) {
@@ -336,10 +395,13 @@ void plan_oneshot_lists(const nuna_topology_t* topo, int num_sms, int nranks, si
     }
 }
 
-static int get_sm_plan(Context* c, int nranks, size_t nvec, int coloc, cudaStream_t stream, SmPlan** out)
+// Looks up (or builds and uploads) the work lists of a shape.  The plan is returned BY VALUE: its device
+// tables stay allocated until nuna_shutdown even when a later probe retires the plan, so a copy taken
+// under the lock stays usable after the lock is dropped.
+static int get_sm_plan(Context* c, int nranks, size_t nvec, int coloc, int domains, cudaStream_t stream, SmPlan* out)
 {
     std::lock_guard<std::mutex> lock(c->mutex);
-    const auto key = std::make_tuple(nranks, nvec, coloc);
+    const auto key = std::make_tuple(nranks, nvec, coloc, domains);
     auto it = c->sm_plans.find(key);
     if (it == c->sm_plans.end()) {
         cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
@@ -349,7 +411,7 @@ static int get_sm_plan(Context* c, int nranks, size_t nvec, int coloc, cudaStrea
         const size_t ntiles = ceil_div(nvec, lanes);
         std::vector<std::vector<unsigned>> lists;
         plan_oneshot_lists(c->have_topology ? &c->topology : nullptr, c->num_sms, nranks, ntiles, lanes * 16,
-                           ntiles <= kGenericPlanTiles, lists);
+                           ntiles <= kGenericPlanTiles, domains, lists);
         std::vector<unsigned> off((size_t)c->num_sms + 1, 0), tiles;
         tiles.reserve(ntiles);
         for (int s = 0; s < c->num_sms; ++s) {
@@ -379,13 +441,13 @@ static int get_sm_plan(Context* c, int nranks, size_t nvec, int coloc, cudaStrea
         pl.ctl = d + cur0 + 2 * (size_t)c->num_sms;
         it = c->sm_plans.emplace(key, pl).first;
     }
-    *out = &it->second;
+    *out = it->second;
     return NUNA_OK;
 }
 
-static int coloc_for(const Context* c, int nranks)
+static int coloc_for(const Options& o, int nranks)
 {
-    int coloc = c->coloc_override > 0 ? c->coloc_override : 8;
+    int coloc = o.coloc > 0 ? o.coloc : 8;
     while (coloc > 1 && coloc / 2 >= nranks) coloc >>= 1;
     return coloc >= 8 ? 8 : coloc >= 4 ? 4 : 2;
 }
@@ -394,156 +456,208 @@ static int coloc_for(const Context* c, int nranks)
 int prepare_oneshot(Context* c, int nranks, int dtype, size_t count, unsigned flags)
 {
     if ((flags & NUNA_PLACE_MASK) == NUNA_PLACE_AWARE && (flags & NUNA_PLACE_SM_LISTS)) {
-        SmPlan* pl = nullptr;
-        return get_sm_plan(c, nranks, count / elems_per_vec(dtype), coloc_for(c, nranks), (cudaStream_t)0, &pl);
+        const Options o = snapshot(c);
+        SmPlan pl;
+        return get_sm_plan(c, nranks, count / elems_per_vec(dtype), coloc_for(o, nranks), o.domains, (cudaStream_t)0, &pl);
     }
     return NUNA_OK;
 }
 
 template <int N, int C, int DT>
-static int launch_sm_lists(Context* c, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
+static int launch_sm_lists(Context* c, const Options& o, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
 {
-    static int occ = 0;
     auto k = k_oneshot_sm<N, C, DT>;
-    SmPlan* pl = nullptr;
-    const int st = get_sm_plan(c, N, count / Elem<DT>::kElems, C, stream, &pl);
+    SmPlan pl;
+    const int st = get_sm_plan(c, N, count / Elem<DT>::kElems, C, o.domains, stream, &pl);
     if (st != NUNA_OK) return st;
     SmLists sl;
-    sl.off = pl->off; sl.tiles = pl->tiles; sl.cursor = pl->cursor; sl.present = pl->present; sl.ctl = pl->ctl;
-    sl.nonempty = pl->nonempty; sl.num_sms = c->num_sms;
-    const size_t cap = (size_t)c->num_sms * (size_t)occupancy(c, k, &occ);
-    const unsigned grid = (unsigned)std::min(cap, std::max<size_t>((size_t)c->num_sms, (size_t)pl->total));
+    sl.off = pl.off; sl.tiles = pl.tiles; sl.cursor = pl.cursor; sl.present = pl.present; sl.ctl = pl.ctl;
+    sl.nonempty = pl.nonempty; sl.num_sms = c->num_sms;
+    const size_t cap = (size_t)c->num_sms * (size_t)NUNA_OCC(k);
+    const unsigned grid = (unsigned)std::min(cap, std::max<size_t>((size_t)c->num_sms, (size_t)pl.total));
     const unsigned blocks_per_sm = (unsigned)std::max<size_t>(1, grid / (size_t)c->num_sms);
     return launch(k, grid, stream, mode, p, count, sl, blocks_per_sm);
 }
 
 template <int N, int DT>
-static int launch_cluster(Context* c, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
+static int launch_cluster(const Options& o, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
 {
     auto k = k_oneshot_cluster<N, DT>;
     const size_t nvec = count / Elem<DT>::kElems;
     const size_t ntiles = std::max<size_t>(1, ceil_div(nvec, (size_t)kThreads));
     size_t clusters = std::min<size_t>(ntiles, (size_t)1 << 20);
-    if (c->blocks_override > 0) clusters = std::max<size_t>(1, std::min<size_t>(clusters, (size_t)c->blocks_override / N));
+    if (o.blocks > 0) clusters = std::max<size_t>(1, std::min<size_t>(clusters, (size_t)o.blocks / N));
     t_cluster_dim = N;
     return launch(k, (unsigned)(clusters * N), stream, mode, p, count, ntiles);
 }
 
 template <int N, int C, int DT>
-static int launch_group(Context* c, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
+static int launch_group(Context* c, const Options& o, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
 {
-    static int occ = 0;
     auto k = k_oneshot_group<N, C, DT>;
     const size_t nvec = count / Elem<DT>::kElems;
     const size_t ntiles = ceil_div(nvec, (size_t)(kThreads / C));
     const size_t nitems = std::max<size_t>(ntiles * ((N + C - 1) / C), (count % Elem<DT>::kElems) ? (size_t)N : 0);
-    const unsigned grid = pick_grid(c, nitems, occupancy(c, k, &occ));
+    const unsigned grid = pick_grid(c, o, nitems, NUNA_OCC(k));
     return launch(k, grid, stream, mode, p, count, ntiles);
+}
+
+// Staged group kernel: one tile per block.  Tile size (vectors per source): large enough that a tile's
+// N slices amortise the copy set-up, small enough that a mid-sized message still gives every SM several
+// blocks; 32 KiB of shared memory per block at most.
+template <int N, int DT>
+static int launch_stage(Context* c, const Options& o, const RankPtrs& p, size_t count, unsigned flags, unsigned mode,
+                        cudaStream_t stream)
+{
+    auto k = k_oneshot_stage<N, DT>;
+    constexpr unsigned kLanes = kThreads / pow2_at_least(N);
+    const size_t nvec = count / Elem<DT>::kElems;
+    // measured at 8 ranks (cold): 4 KiB tiles up to 512 KiB per rank, 8 KiB to 4 MiB, 16 KiB to 16 MiB, 32 KiB beyond
+    const size_t bytes = count * (size_t)Elem<DT>::kBytes;
+    unsigned tile_bytes = bytes <= ((size_t)512 << 10) ? 4096u : bytes <= ((size_t)4 << 20) ? 8192u
+                        : bytes <= ((size_t)16 << 20) ? 16384u : 32768u;
+    unsigned tv = tile_bytes / 16u / (unsigned)pow2_at_least(N);
+    if (o.stage_vecs > 0) tv = (unsigned)o.stage_vecs;
+    tv = std::max(kLanes, std::min(tv, 2048u / N)) / kLanes * kLanes;     // a multiple of the row width, <= 32 KiB per tile
+    const size_t ntiles = ceil_div(nvec, (size_t)tv);
+    const size_t grid = std::max<size_t>(ntiles, (count % Elem<DT>::kElems) ? 1 : 0);
+    t_dyn_smem = (unsigned)N * tv * 16u;
+    return launch(k, (unsigned)std::max<size_t>(1, grid), stream, mode, p, count, tv,
+                  (flags & NUNA_HINT_RESIDENT) ? 0 : 1, &c->bw->status, o.timeout_ns);
 }
 
 int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t count, unsigned flags, cudaStream_t stream)
 {
+    const Options o = snapshot(c);
     const size_t bytes = count * elem_size(dtype);                   // per rank
     const size_t epv = elems_per_vec(dtype);
     const unsigned mode = launch_mode(flags, bytes * (size_t)nranks);
     const size_t nvec = count / epv;
     const unsigned place = flags & NUNA_PLACE_MASK;
-    if (place == NUNA_PLACE_AWARE || (place == NUNA_PLACE_AUTO && aware_pays_off(c, nranks, bytes, flags))) {
+    OneShotKernel which = OneShotKernel::RoundRobin;
+    if (place == NUNA_PLACE_AWARE) which = (flags & NUNA_PLACE_STAGED) ? OneShotKernel::Staged : OneShotKernel::Group;
+    else if (place == NUNA_PLACE_AUTO) which = auto_kernel(c, o, nranks, bytes, flags);
+    if (which == OneShotKernel::Staged) {
+        return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
+            constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
+            return launch_stage<N, DT>(c, o, p, count, flags, (flags & NUNA_LAUNCH_PDL) ? kLaunchPdl : kLaunchPlain, stream);
+        });
+    }
+    if (which == OneShotKernel::Group) {
         // co-location factor: C destinations of a tile share a block (C <= N rounded up to a power of two)
-        const int coloc = coloc_for(c, nranks);
-        if ((flags & NUNA_PLACE_CLUSTER) && nranks >= 2 && nranks <= 8) {
+        const int coloc = coloc_for(o, nranks);
+        if (place == NUNA_PLACE_AWARE && (flags & NUNA_PLACE_CLUSTER) && nranks >= 2 && nranks <= 8) {
             return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
                 constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
-                if constexpr (N >= 2 && N <= 8) return launch_cluster<N, DT>(c, p, count, mode, stream);
+                if constexpr (N >= 2 && N <= 8) return launch_cluster<N, DT>(o, p, count, mode, stream);
                 else return NUNA_ERR_INVALID_ARG;
             });
         }
-        if (flags & NUNA_PLACE_SM_LISTS) {
+        if (place == NUNA_PLACE_AWARE && (flags & NUNA_PLACE_SM_LISTS)) {
             return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
                 constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
-                if (coloc >= 8) return launch_sm_lists<N, 8, DT>(c, p, count, mode, stream);
-                if (coloc >= 4) return launch_sm_lists<N, 4, DT>(c, p, count, mode, stream);
-                return launch_sm_lists<N, 2, DT>(c, p, count, mode, stream);
+                if (coloc >= 8) return launch_sm_lists<N, 8, DT>(c, o, p, count, mode, stream);
+                if (coloc >= 4) return launch_sm_lists<N, 4, DT>(c, o, p, count, mode, stream);
+                return launch_sm_lists<N, 2, DT>(c, o, p, count, mode, stream);
             });
         }
         return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
             constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
-            if (coloc >= 8) return launch_group<N, 8, DT>(c, p, count, mode, stream);
-            if (coloc >= 4) return launch_group<N, 4, DT>(c, p, count, mode, stream);
-            return launch_group<N, 2, DT>(c, p, count, mode, stream);
+            if (coloc >= 8) return launch_group<N, 8, DT>(c, o, p, count, mode, stream);
+            if (coloc >= 4) return launch_group<N, 4, DT>(c, o, p, count, mode, stream);
+            return launch_group<N, 2, DT>(c, o, p, count, mode, stream);
         });
     }
-    return dispatch(nranks, pick_unroll(c, nranks), dtype, [&](auto n_, auto u_, auto d_) -> int {
+    return dispatch(nranks, pick_unroll(o, nranks), dtype, [&](auto n_, auto u_, auto d_) -> int {
         NUNA_NUD(n_, u_, d_);
-        static int occ = 0;
         auto k = k_oneshot_rr<N, U, DT>;
         const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
         const size_t nitems = std::max<size_t>(ntiles * N, (count % epv) ? (size_t)N : 0);
         // one resident wave while the message is small enough for latency to matter, four beyond
-        const unsigned grid = pick_grid(c, nitems, occupancy(c, k, &occ), bytes >= ((size_t)8 << 20) ? 4 : 1);
+        const unsigned grid = pick_grid(c, o, nitems, NUNA_OCC(k), bytes >= ((size_t)8 << 20) ? 4 : 1);
         return launch(k, grid, stream, mode, p, count, ntiles);
     });
 }
 
-// Launches the flag-barrier two-shot on explicit scratch / barrier storage (the context's, or the
-// fixed arrays of the allocation-free entry point).
-static int launch_twoshot_fused(int num_sms, int blocks_override, const RankPtrs& p, int nranks, int dtype, size_t count,
-                                int u, uint4* scratch, BarrierWords* bw, unsigned long long timeout_ns,
-                                cudaStream_t stream)
+// Launches the flag-synchronised two-shot on explicit scratch / flag / control storage (the context's, or
+// the fixed arrays of the allocation-free entry point): one block per work item, tiles + lead blocks.
+// tv = 0 picks the tile size by message size.  min_tv is the smallest tile the flag array was sized for.
+int launch_twoshot_flags(int num_sms, int blocks_override, const RankPtrs& p, int nranks, int dtype, size_t count,
+                         unsigned tv, unsigned min_tv, uint4* scratch, unsigned* tile_flags, BarrierWords* bw,
+                         unsigned long long timeout_ns, bool pdl, unsigned wait_bias, cudaStream_t stream)
 {
-    // chunk = ceil(count / N) rounded up to whole vectors
-    const size_t chunk_vec = ceil_div(ceil_div(count, (size_t)nranks), elems_per_vec(dtype));
-    return dispatch(nranks, u, dtype, [&](auto n_, auto u_, auto d_) -> int {
-        NUNA_NUD(n_, u_, d_);
-        static int occ = 0;
-        auto k = k_twoshot_fused<N, U, DT>;
-        const size_t tiles_per_chunk = ceil_div(chunk_vec, (size_t)kThreads * U);
-        // every block must be resident for the flag barrier: never more than the device holds at once
-        size_t cap = (size_t)num_sms * (size_t)occupancy(nullptr, k, &occ);
-        if (blocks_override > 0) cap = std::min<size_t>(cap, (size_t)blocks_override);
-        const unsigned grid = (unsigned)std::max<size_t>(1, std::min(tiles_per_chunk * N, cap));
-        return launch(k, grid, stream, kLaunchCooperative, p, scratch, count, chunk_vec, bw, timeout_ns);
+    const size_t bytes = count * elem_size(dtype);
+    const size_t nvec = count / elems_per_vec(dtype);
+    if (tv == 0) {
+        // tile bytes across all N sources: small tiles while the message is small (more blocks, less latency
+        // per tile), up to 32 KiB once there are plenty of tiles
+        const size_t src_bytes = bytes * (size_t)nranks;
+        const unsigned tile_src = src_bytes <= ((size_t)1 << 20) ? 4096u : src_bytes <= ((size_t)8 << 20) ? 8192u
+                                : src_bytes <= ((size_t)64 << 20) ? 16384u : 32768u;
+        tv = tile_src / 16u / (unsigned)nranks;
+    }
+    tv = std::max(min_tv, std::min(tv, 2048u / (unsigned)nranks));
+    tv = std::max(1u, tv / 8u * 8u);
+    if (tv < min_tv) tv = min_tv;
+    const size_t ntiles = std::max<size_t>(1, ceil_div(nvec, (size_t)tv));
+    unsigned lead_max = (unsigned)num_sms * 8u;
+    if (blocks_override > 0) lead_max = (unsigned)std::max(1, blocks_override);
+    const size_t lead = std::min<size_t>(ntiles, lead_max);
+    const unsigned grid = (unsigned)(ntiles + lead);
+    return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
+        constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
+        auto k = k_twoshot_flags<N, DT>;
+        t_dyn_smem = (unsigned)N * tv * 16u;
+        return launch(k, grid, stream, pdl ? kLaunchPdl : kLaunchPlain, p, scratch, tile_flags, count, tv, lead_max, bw,
+                      timeout_ns, wait_bias);
     });
 }
 
 int launch_twoshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t count, unsigned flags, cudaStream_t stream)
 {
+    const Options o = snapshot(c);
     const size_t epv = elems_per_vec(dtype);
     const unsigned mode = launch_mode(flags);
     const size_t nvec = count / epv;
     if (flags & NUNA_TWOSHOT_PUT) {
-        return dispatch(nranks, pick_unroll(c, nranks), dtype, [&](auto n_, auto u_, auto d_) -> int {
+        return dispatch(nranks, pick_unroll(o, nranks), dtype, [&](auto n_, auto u_, auto d_) -> int {
             NUNA_NUD(n_, u_, d_);
-            static int occ = 0;
             auto k = k_twoshot_put<N, U, DT>;
             const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
-            const unsigned grid = pick_grid(c, std::max<size_t>(ntiles, 1), occupancy(c, k, &occ), 0);
+            const unsigned grid = pick_grid(c, o, std::max<size_t>(ntiles, 1), NUNA_OCC(k), 0);
             return launch(k, grid, stream, mode, p, count, ntiles);
         });
     }
-    return launch_twoshot_fused(c->num_sms, c->blocks_override, p, nranks, dtype, count, pick_unroll(c, nranks),
-                                reinterpret_cast<uint4*>(c->scratch), c->bw, c->timeout_ns, stream);
+    uint4* scratch;
+    unsigned* tile_flags;
+    {
+        std::lock_guard<std::mutex> lock(c->mutex);
+        scratch = reinterpret_cast<uint4*>(c->scratch);
+        tile_flags = c->flags;
+    }
+    return launch_twoshot_flags(c->num_sms, o.blocks, p, nranks, dtype, count, (unsigned)std::max(0, o.twoshot_vecs), kMinFlagTileVec,
+                                scratch, tile_flags, c->bw, o.timeout_ns, (flags & NUNA_LAUNCH_PDL) != 0, 0u, stream);
 }
 
 int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, int dtype, size_t shard, unsigned flags,
                           cudaStream_t stream)
 {
+    const Options o = snapshot(c);
     const size_t epv = elems_per_vec(dtype);
     const unsigned mode = launch_mode(flags);
     if (shard % epv) {
-        const unsigned grid = pick_grid(c, ceil_div(shard * nranks, kThreads), 8);
+        const unsigned grid = pick_grid(c, o, ceil_div(shard * nranks, kThreads), 8);
         return dispatch(nranks, 1, dtype, [&](auto n_, auto u_, auto d_) -> int {
             NUNA_NUD(n_, u_, d_);
             return launch(k_reduce_scatter_scalar<N, DT>, grid, stream, mode, p, shard);
         });
     }
     const size_t shard_vec = shard / epv;
-    return dispatch(nranks, pick_unroll(c, nranks), dtype, [&](auto n_, auto u_, auto d_) -> int {
+    return dispatch(nranks, pick_unroll(o, nranks), dtype, [&](auto n_, auto u_, auto d_) -> int {
         NUNA_NUD(n_, u_, d_);
-        static int occ = 0;
         auto k = k_reduce_scatter<N, U, DT>;
         const size_t tiles = ceil_div(shard_vec, (size_t)kThreads * U);
-        const unsigned grid = pick_grid(c, tiles * N, occupancy(c, k, &occ), 0);
+        const unsigned grid = pick_grid(c, o, tiles * N, NUNA_OCC(k), 0);
         return launch(k, grid, stream, mode, p, shard_vec, tiles);
     });
 }
@@ -552,14 +666,14 @@ int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, int dtype, 
 // them, otherwise on 16-bit units (every element type is a multiple of that).
 int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard_bytes, unsigned flags, cudaStream_t stream)
 {
+    const Options o = snapshot(c);
     const unsigned mode = launch_mode(flags);
     if (shard_bytes % 16) {
         const size_t shard16 = shard_bytes / 2;
-        const unsigned grid = pick_grid(c, ceil_div(shard16 * nranks, kThreads), 8);
+        const unsigned grid = pick_grid(c, o, ceil_div(shard16 * nranks, kThreads), 8);
         return launch(k_allgather_scalar, grid, stream, mode, p, nranks, shard16);
     }
     const size_t shard_vec = shard_bytes / 16;
-    static int occ = 0;
     // One block per (rank, tile) storing to all N destinations.  Splitting a tile's destinations over
     // several blocks (dsplit > 1) was measured slower at every size tried (16 x 64 KiB: 4.4 us with 1,
     // 5.4 us with 8): the stores, not the block count, are the limit.
@@ -567,25 +681,72 @@ int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard_byt
     const int dsplit = 1;
     auto k = k_allgather<U>;
     const size_t tiles = ceil_div(shard_vec, (size_t)kThreads * U);
-    const unsigned grid = pick_grid(c, tiles * nranks * dsplit, occupancy(c, k, &occ), 0);
+    const unsigned grid = pick_grid(c, o, tiles * nranks * dsplit, NUNA_OCC(k), 0);
     return launch(k, grid, stream, mode, p, nranks, shard_vec, tiles, dsplit);
 }
 
 int launch_alltoall(Context* c, const RankPtrs& p, int nranks, size_t block_bytes, unsigned flags, cudaStream_t stream)
 {
+    const Options o = snapshot(c);
     const unsigned mode = launch_mode(flags);
     if (block_bytes % 16) {
         const size_t block16 = block_bytes / 2;
-        const unsigned grid = pick_grid(c, ceil_div(block16 * nranks * nranks, kThreads), 8);
+        const unsigned grid = pick_grid(c, o, ceil_div(block16 * nranks * nranks, kThreads), 8);
         return launch(k_alltoall_scalar, grid, stream, mode, p, nranks, block16);
     }
     const size_t block_vec = block_bytes / 16;
-    static int occ = 0;
     constexpr int U = 2;
     auto k = k_alltoall<U>;
     const size_t tiles = ceil_div(block_vec, (size_t)kThreads * U);
-    const unsigned grid = pick_grid(c, tiles * nranks * nranks, occupancy(c, k, &occ), 0);
+    const unsigned grid = pick_grid(c, o, tiles * nranks * nranks, NUNA_OCC(k), 0);
     return launch(k, grid, stream, mode, p, nranks, block_vec, tiles);
+}
+
+// ---- single-kernel chain ---------------------------------------------------------------------------------
+
+// One cluster runs the whole chain, so it pays only while a node's work is small next to a kernel launch.
+constexpr size_t kChainPersistentMaxBytes = (size_t)128 << 10;     // per rank
+
+bool chain_persistent_supported(const Context* c, int nsets, int nranks, int dtype, size_t count)
+{
+    (void)c;
+    return nsets >= 1 && nsets <= kMaxChainSets && nranks >= 1 && count * elem_size(dtype) <= ((size_t)4 << 20);
+}
+
+bool chain_persistent_pays_off(int dtype, size_t count) { return count * elem_size(dtype) <= kChainPersistentMaxBytes; }
+
+int launch_chain_persistent(Context* c, const ChainSets& sets, int nsets, int nnodes, int nranks, int dtype, size_t count,
+                            cudaStream_t stream)
+{
+    (void)c;
+    return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
+        constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
+        auto k = k_chain_persistent<N, DT>;
+        // sixteen blocks per cluster need the non-portable opt-in; fall back to the portable eight
+        static std::atomic<int> cluster_size[kMaxDevices];
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+        int cs = cluster_size[dev].load(std::memory_order_relaxed);
+        if (cs == 0) {
+            cs = 8;
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(16, 1, 1);
+                cfg.blockDim = dim3(kThreads, 1, 1);
+                cudaLaunchAttribute at;
+                at.id = cudaLaunchAttributeClusterDimension;
+                at.val.clusterDim.x = 16; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+                cfg.attrs = &at;
+                cfg.numAttrs = 1;
+                int nclusters = 0;
+                if (cudaOccupancyMaxActiveClusters(&nclusters, k, &cfg) == cudaSuccess && nclusters >= 1) cs = 16;
+            }
+            cudaGetLastError();
+            cluster_size[dev].store(cs, std::memory_order_relaxed);
+        }
+        t_cluster_dim = (unsigned)cs;
+        return launch(k, (unsigned)cs, stream, kLaunchPlain, sets, nsets, nnodes, count);
+    });
 }
 
 }  // namespace nuna
@@ -611,11 +772,14 @@ int nuna_set_option(int option, long long value)
     if (st != NUNA_OK) return st;
     std::lock_guard<std::mutex> lock(c->mutex);
     switch (option) {
-        case NUNA_OPT_BLOCKS: c->blocks_override = (int)std::min<long long>(value, 1 << 22); break;
-        case NUNA_OPT_UNROLL: c->unroll_override = (int)value; break;
-        case NUNA_OPT_COLOC: c->coloc_override = (int)value; break;
-        case NUNA_OPT_AUTO_MIN_BYTES: c->auto_min_bytes = value ? (size_t)value : ((size_t)64 << 10); break;
-        case NUNA_OPT_TIMEOUT_MS: c->timeout_ns = (unsigned long long)(value ? value : 1000) * 1000000ull; break;
+        case NUNA_OPT_BLOCKS: c->opt.blocks = (int)std::min<long long>(value, 1 << 22); break;
+        case NUNA_OPT_UNROLL: c->opt.unroll = (int)value; break;
+        case NUNA_OPT_COLOC: c->opt.coloc = (int)value; break;
+        case NUNA_OPT_AUTO_MIN_BYTES: c->opt.auto_min_bytes = value ? (size_t)value : ((size_t)64 << 10); break;
+        case NUNA_OPT_TIMEOUT_MS: c->opt.timeout_ns = (unsigned long long)(value ? value : 1000) * 1000000ull; break;
+        case NUNA_OPT_DOMAINS: c->opt.domains = (int)std::min<long long>(value, NUNA_MAX_SMS); break;
+        case NUNA_OPT_STAGE_VECS: c->opt.stage_vecs = (int)std::min<long long>(value, 4096); break;
+        case NUNA_OPT_TWOSHOT_VECS: c->opt.twoshot_vecs = (int)std::min<long long>(value, 4096); break;
         default: return NUNA_ERR_INVALID_ARG;
     }
     return NUNA_OK;
@@ -624,6 +788,7 @@ int nuna_set_option(int option, long long value)
 int nuna_allreduce_oneshot(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
                            unsigned flags, void* stream)
 {
+    if (has_chain_bits(flags)) return NUNA_ERR_INVALID_ARG;
     int st = check_args(src, dst, nranks, count, count, dtype, flags & ~NUNA_TWOSHOT_PUT, true);
     if (st != NUNA_OK || count == 0) return st;
     if (flags & NUNA_TWOSHOT_PUT) return NUNA_ERR_INVALID_ARG;
@@ -635,6 +800,7 @@ int nuna_allreduce_oneshot(const void* const* src, void* const* dst, int nranks,
 int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
                            unsigned flags, void* stream)
 {
+    if (has_chain_bits(flags)) return NUNA_ERR_INVALID_ARG;
     int st = check_args(src, dst, nranks, count, count, dtype, flags, true);
     if (st != NUNA_OK || count == 0) return st;
     Context* c = nullptr;
@@ -642,7 +808,7 @@ int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
     if (!(flags & NUNA_TWOSHOT_PUT)) {
         std::lock_guard<std::mutex> lock(c->mutex);
         const size_t need = (count * elem_size(dtype) + 15) & ~(size_t)15;
-        if (need > c->scratch_bytes) {
+        if (need > c->scratch_bytes || !c->scratch) {
             cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
             if (cudaStreamIsCapturing((cudaStream_t)stream, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone)
                 return NUNA_ERR_CAPTURING;             // growing the scratch allocates: call nuna_init first
@@ -655,20 +821,26 @@ int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
 int nuna_allreduce(const void* const* src, void* const* dst, int nranks, size_t count, int dtype, unsigned flags,
                    void* stream)
 {
-    // Crossover measured on B200, cold and L2-resident, with dependent launch: the one-shot's N-fold
-    // re-reads cost more the more ranks there are, so it wins up to 1 MiB per rank at 2 ranks,
-    // 512 KiB at 4, 128 KiB at 8 and 64 KiB at 16.
+    // Crossover measured on B200, cold and L2-resident: the one-shot's N-fold re-reads cost more the
+    // more ranks there are, so its single step wins up to 1 MiB per rank at 2 ranks, 512 KiB at 4,
+    // 128 KiB at 8 and 64 KiB at 16.  Beyond it the put form of the two-shot is the fastest kernel at every
+    // size; the flag-synchronised form is used instead when the caller asks for it (NUNA_TWOSHOT_SYNC),
+    // from the size where it beats the one-shot (measured per rank count, kSyncFactor x the put crossover).
     const size_t bytes = count * elem_size(dtype);
     const size_t limit = nranks <= 2 ? ((size_t)1 << 20) : nranks <= 4 ? ((size_t)512 << 10)
                        : nranks <= 8 ? ((size_t)128 << 10) : ((size_t)64 << 10);
-    if (nranks <= 1 || bytes <= limit)
-        return nuna_allreduce_oneshot(src, dst, nranks, count, dtype, flags & ~NUNA_TWOSHOT_PUT, stream);
-    return nuna_allreduce_twoshot(src, dst, nranks, count, dtype, flags, stream);
+    constexpr size_t kSyncFactor = 8;
+    const bool sync_form = (flags & NUNA_TWOSHOT_SYNC) && !(flags & NUNA_TWOSHOT_PUT);
+    const unsigned base = flags & ~(NUNA_TWOSHOT_SYNC | NUNA_TWOSHOT_PUT);
+    if (nranks <= 1 || bytes <= (sync_form ? limit * kSyncFactor : limit))
+        return nuna_allreduce_oneshot(src, dst, nranks, count, dtype, base, stream);
+    return nuna_allreduce_twoshot(src, dst, nranks, count, dtype, sync_form ? base : (base | NUNA_TWOSHOT_PUT), stream);
 }
 
 int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks, size_t shard_count, int dtype,
                         unsigned flags, void* stream)
 {
+    if (has_chain_bits(flags)) return NUNA_ERR_INVALID_ARG;
     if (nranks >= 1 && nranks <= NUNA_MAX_RANKS && shard_count > ((size_t)1 << 40) / (size_t)nranks)
         return NUNA_ERR_TOO_LARGE;
     int st = check_args(src, dst, nranks, shard_count * (size_t)(nranks > 0 ? nranks : 0), shard_count, dtype,
@@ -683,6 +855,7 @@ int nuna_reduce_scatter(const void* const* src, void* const* dst, int nranks, si
 int nuna_allgather(const void* const* src, void* const* dst, int nranks, size_t shard_count, int dtype,
                    unsigned flags, void* stream)
 {
+    if (has_chain_bits(flags)) return NUNA_ERR_INVALID_ARG;
     if (nranks >= 1 && nranks <= NUNA_MAX_RANKS && shard_count > ((size_t)1 << 40) / (size_t)nranks)
         return NUNA_ERR_TOO_LARGE;
     int st = check_args(src, dst, nranks, shard_count, shard_count * (size_t)(nranks > 0 ? nranks : 0), dtype,
@@ -697,6 +870,7 @@ int nuna_allgather(const void* const* src, void* const* dst, int nranks, size_t 
 int nuna_alltoall(const void* const* src, void* const* dst, int nranks, size_t block_count, int dtype,
                   unsigned flags, void* stream)
 {
+    if (has_chain_bits(flags)) return NUNA_ERR_INVALID_ARG;
     if (nranks >= 1 && nranks <= NUNA_MAX_RANKS && block_count > ((size_t)1 << 40) / (size_t)nranks)
         return NUNA_ERR_TOO_LARGE;
     const size_t per_rank = block_count * (size_t)(nranks > 0 ? nranks : 0);
@@ -711,12 +885,13 @@ int nuna_alltoall(const void* const* src, void* const* dst, int nranks, size_t b
 int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
                         unsigned flags, int two_shot)
 {
+    if (has_chain_bits(flags)) return NUNA_ERR_INVALID_ARG;
     int st = check_args(src, dst, nranks, count, count, dtype, flags, false);
     if (st != NUNA_OK || count == 0) return st;
     if (!two_shot && (flags & NUNA_TWOSHOT_PUT)) return NUNA_ERR_INVALID_ARG;
     Context* c = nullptr;
     if ((st = get_context(&c)) != NUNA_OK) return st;
-    std::lock_guard<std::mutex> lock(c->mutex);
+    std::lock_guard<std::mutex> lock(c->host_mutex);       // staging buffers and the private stream: one call at a time
     const size_t bytes = count * elem_size(dtype);
     if (!c->stream && cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking) != cudaSuccess) return NUNA_ERR_CUDA;
 
@@ -755,7 +930,10 @@ int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks, si
         if (cudaMalloc(&c->staging, need) != cudaSuccess) return NUNA_ERR_CUDA;
         c->staging_bytes = need;
     }
-    if (two_shot && !(flags & NUNA_TWOSHOT_PUT) && (st = ensure_scratch(c, slot)) != NUNA_OK) return st;
+    if (two_shot && !(flags & NUNA_TWOSHOT_PUT)) {
+        std::lock_guard<std::mutex> inner(c->mutex);
+        if ((st = ensure_scratch(c, slot)) != NUNA_OK) return st;
+    }
     const void* dsrc[NUNA_MAX_RANKS];
     void* ddst[NUNA_MAX_RANKS];
     char* base = static_cast<char*>(c->staging);
@@ -784,8 +962,12 @@ int nuna_device_status(int* out)
     if (cudaDeviceSynchronize() != cudaSuccess) return NUNA_ERR_CUDA;
     BarrierWords h;
     if (cudaMemcpy(&h, c->bw, sizeof h, cudaMemcpyDeviceToHost) != cudaSuccess) return NUNA_ERR_CUDA;
-    *out = (int)h.status;
-    if (h.status != 0) return init_barrier_words(c);
+    unsigned worst = h.status;
+    if (h.status != 0 && (st = rewind_barrier_words(c->bw, h)) != NUNA_OK) return st;
+    // the allocation-free entry point keeps its own words in the library's fixed arrays
+    unsigned static_status = 0;
+    if ((st = static_status_read_and_clear(&static_status)) != NUNA_OK) return st;
+    *out = (int)std::max(worst, static_status);
     return NUNA_OK;
 }
 
@@ -824,6 +1006,7 @@ int nuna_shutdown(void)
     cudaDeviceSynchronize();
     if (c->bw) cudaFree(c->bw);
     if (c->scratch) cudaFree(c->scratch);
+    for (void* d : c->retired_scratch) cudaFree(d);
     if (c->staging) cudaFree(c->staging);
     if (c->stream) cudaStreamDestroy(c->stream);
     for (auto& kv : c->sm_plans) cudaFree(kv.second.base);
@@ -836,11 +1019,11 @@ int nuna_shutdown(void)
 /* Test hook: the per-SM work lists planned for a one-shot of `ntiles` tiles under `topo` (NULL = no probe),
  * by the general planner (generic != 0) or the closed form.  off: [num_sms + 1], tiles: [ntiles].          */
 int nuna_debug_plan_oneshot(const nuna_topology_t* topo, int num_sms, int nranks, size_t ntiles, size_t tile_bytes,
-                            int generic, unsigned* off, unsigned* tiles)
+                            int generic, int domains, unsigned* off, unsigned* tiles)
 {
-    if (num_sms < 1 || nranks < 1 || nranks > NUNA_MAX_RANKS || !off || !tiles) return NUNA_ERR_INVALID_ARG;
+    if (num_sms < 1 || nranks < 1 || nranks > NUNA_MAX_RANKS || !off || !tiles || domains < 0) return NUNA_ERR_INVALID_ARG;
     std::vector<std::vector<unsigned>> lists;
-    plan_oneshot_lists(topo, num_sms, nranks, ntiles, tile_bytes, generic != 0, lists);
+    plan_oneshot_lists(topo, num_sms, nranks, ntiles, tile_bytes, generic != 0, domains, lists);
     size_t n = 0;
     off[0] = 0;
     for (int s = 0; s < num_sms; ++s) {
@@ -871,6 +1054,28 @@ int nuna_debug_barrier_selftest(unsigned grid, unsigned expected, unsigned timeo
     return st;
 }
 
+/* Test hook: a flag-synchronised two-shot whose consumer items wait for a flag value that nobody publishes
+ * (wait_bias = 1).  Every consumer wait runs out after timeout_ms, the kernel returns, destinations stay
+ * unwritten and the status word latches NUNA_ERR_TIMEOUT -- nothing traps or hangs.                       */
+int nuna_debug_twoshot_unset_flags(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
+                                   unsigned timeout_ms)
+{
+    int st = check_args(src, dst, nranks, count, count, dtype, 0u, true);
+    if (st != NUNA_OK || count == 0) return st;
+    Context* c = nullptr;
+    if ((st = get_context(&c)) != NUNA_OK) return st;
+    uint4* scratch;
+    unsigned* tile_flags;
+    {
+        std::lock_guard<std::mutex> lock(c->mutex);
+        if ((st = ensure_scratch(c, (count * elem_size(dtype) + 15) & ~(size_t)15)) != NUNA_OK) return st;
+        scratch = reinterpret_cast<uint4*>(c->scratch);
+        tile_flags = c->flags;
+    }
+    return launch_twoshot_flags(c->num_sms, 0, make_ptrs(src, dst, nranks), nranks, dtype, count, 0u, kMinFlagTileVec, scratch,
+                                tile_flags, c->bw, (unsigned long long)timeout_ms * 1000000ull, false, 1u, (cudaStream_t)0);
+}
+
 }  // extern "C"
 
 // ---- two-shot allreduce for callers that cannot allocate ------------------------------------------
@@ -884,18 +1089,20 @@ int nuna_debug_barrier_selftest(unsigned grid, unsigned expected, unsigned timeo
 namespace nuna {
 
 static __device__ __align__(256) unsigned char g_static_shard[NUNA_STATIC_MAX_COUNT * 2];
+static __device__ __align__(256) unsigned int g_static_flags[NUNA_STATIC_MAX_COUNT * 2 / (kStaticTileVec * 16) + 1];   // one per tile
 static __device__ __align__(256) BarrierWords g_static_barrier;
 
 struct StaticSetup {
     bool ready = false;
     uint4* shard = nullptr;              // device address of g_static_shard on this device
-    BarrierWords* barrier = nullptr;     // device address of g_static_barrier on this device
+    unsigned* flags = nullptr;           // device address of g_static_flags
+    BarrierWords* barrier = nullptr;     // device address of g_static_barrier
     int num_sms = 0;
 };
 static StaticSetup g_static_setup[kMaxDevices];
 static std::mutex g_static_mutex;
 
-// Once per device: resolve the two symbols and zero the barrier words.  No allocation.
+// Once per device: resolve the symbols and zero the control words and ready flags.  No allocation.
 static int static_setup(StaticSetup** out)
 {
     int dev = -1;
@@ -904,19 +1111,41 @@ static int static_setup(StaticSetup** out)
     StaticSetup& s = g_static_setup[dev];
     if (!s.ready) {
         void* shard = nullptr;
+        void* flags = nullptr;
         void* barrier = nullptr;
         if (cudaGetSymbolAddress(&shard, g_static_shard) != cudaSuccess || !shard) return NUNA_ERR_CUDA;
+        if (cudaGetSymbolAddress(&flags, g_static_flags) != cudaSuccess || !flags) return NUNA_ERR_CUDA;
         if (cudaGetSymbolAddress(&barrier, g_static_barrier) != cudaSuccess || !barrier) return NUNA_ERR_CUDA;
         if (cudaDeviceGetAttribute(&s.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || s.num_sms < 1)
             return NUNA_ERR_CUDA;
-        // the barrier counts arrivals from zero; the shard needs no clearing (written before it is read)
+        // epoch, cursor and departure counter start from zero, and no tile may read as ready; the shard
+        // needs no clearing (every element is written before it is read)
         if (cudaMemset(barrier, 0, sizeof(BarrierWords)) != cudaSuccess) return NUNA_ERR_CUDA;
+        if (cudaMemset(flags, 0, sizeof(g_static_flags)) != cudaSuccess) return NUNA_ERR_CUDA;
         s.shard = static_cast<uint4*>(shard);
+        s.flags = static_cast<unsigned*>(flags);
         s.barrier = static_cast<BarrierWords*>(barrier);
         s.ready = true;
     }
     *out = &s;
     return NUNA_OK;
+}
+
+// For nuna_device_status: the status latched by the allocation-free entry point on the current device
+// (0 if that entry point was never used here).  A latched timeout leaves cursor and departure counter in
+// an undefined state, so the control words are zeroed again; the device is idle (the caller synchronised).
+static int static_status_read_and_clear(unsigned* out)
+{
+    *out = 0;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return NUNA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticSetup& s = g_static_setup[dev];
+    if (!s.ready) return NUNA_OK;
+    BarrierWords h;
+    if (cudaMemcpy(&h, s.barrier, sizeof h, cudaMemcpyDeviceToHost) != cudaSuccess) return NUNA_ERR_CUDA;
+    *out = h.status;
+    return h.status != 0 ? rewind_barrier_words(s.barrier, h) : NUNA_OK;
 }
 
 }  // namespace nuna
@@ -934,7 +1163,7 @@ extern "C" int nuna_allreduce_twoshot_static(const void* const* src, void* const
     }
     StaticSetup* s = nullptr;
     if ((st = static_setup(&s)) != NUNA_OK) return st;
-    const int u = 1;
-    return launch_twoshot_fused(s->num_sms, 0, make_ptrs(src, dst, nranks), nranks, dtype, count, u, s->shard, s->barrier,
-                                1000000000ull, (cudaStream_t)stream);
+    // tiles of 4 KiB per source (the fixed flag array has one word per 4 KiB of the shard), fewer vectors for many ranks
+    return launch_twoshot_flags(s->num_sms, 0, make_ptrs(src, dst, nranks), nranks, dtype, count, kStaticTileVec, kStaticTileVec,
+                                s->shard, s->flags, s->barrier, 1000000000ull, false, 0u, (cudaStream_t)stream);
 }

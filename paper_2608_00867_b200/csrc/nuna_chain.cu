@@ -1,4 +1,5 @@
-// CUDA-graph chain of back-to-back allreduces: one decode step's per-layer collectives.
+// Chain of back-to-back allreduces: one decode step's per-layer collectives, as a CUDA graph of one
+// kernel per node or, for small nodes, as a single kernel (k_chain_persistent) that loops over the nodes.
 //
 // The nodes are captured once from a private stream and replayed with one graph launch, so control
 // never returns to the host inside a step.  Node k works on buffer set k mod nsets and may not
@@ -12,7 +13,12 @@
 namespace nuna {
 
 struct Chain {
-    cudaGraphExec_t exec = nullptr;
+    cudaGraphExec_t exec = nullptr;      // graph form: one kernel node per allreduce
+    bool persistent = false;             // single-kernel form: the fields below
+    ChainSets sets = {};
+    int nsets = 0, nranks = 0, dtype = 0;
+    size_t count = 0;
+    Context* ctx = nullptr;
     int device = -1;
     int nnodes = 0;
 };
@@ -40,6 +46,29 @@ int nuna_chain_create(const void* const* src_sets, void* const* dst_sets, int ns
     Context* c = nullptr;
     int st = get_context(&c);
     if (st != NUNA_OK) return st;
+    if ((flags & NUNA_CHAIN_PERSISTENT) && (flags & NUNA_CHAIN_GRAPH)) return NUNA_ERR_INVALID_ARG;
+    const bool can_persist = !two_shot && chain_persistent_supported(c, nsets, nranks, dtype, count);
+    if ((flags & NUNA_CHAIN_PERSISTENT) && !can_persist) return NUNA_ERR_INVALID_ARG;
+    if (can_persist && !(flags & NUNA_CHAIN_GRAPH) &&
+        ((flags & NUNA_CHAIN_PERSISTENT) || chain_persistent_pays_off(dtype, count))) {
+        Chain* ch = new Chain();
+        ch->persistent = true;
+        ch->device = c->device;
+        ch->ctx = c;
+        ch->nnodes = nnodes;
+        ch->nsets = nsets;
+        ch->nranks = nranks;
+        ch->dtype = dtype;
+        ch->count = count;
+        for (int s = 0; s < nsets; ++s)
+            for (int r = 0; r < nranks; ++r) {
+                ch->sets.s[s].src[r] = reinterpret_cast<const uint4*>(src_sets[(size_t)s * nranks + r]);
+                ch->sets.s[s].dst[r] = reinterpret_cast<uint4*>(dst_sets[(size_t)s * nranks + r]);
+            }
+        *chain_out = ch;
+        return NUNA_OK;
+    }
+    flags &= ~(NUNA_CHAIN_PERSISTENT | NUNA_CHAIN_GRAPH);
     if (two_shot && !(flags & NUNA_TWOSHOT_PUT)) {
         std::lock_guard<std::mutex> lock(c->mutex);
         if ((st = ensure_scratch(c, (count * elem_size(dtype) + 15) & ~(size_t)15)) != NUNA_OK) return st;
@@ -85,7 +114,11 @@ int nuna_chain_create(const void* const* src_sets, void* const* dst_sets, int ns
 int nuna_chain_launch(void* chain, void* stream)
 {
     Chain* ch = static_cast<Chain*>(chain);
-    if (!ch || !ch->exec) return NUNA_ERR_INVALID_ARG;
+    if (!ch) return NUNA_ERR_INVALID_ARG;
+    if (ch->persistent)
+        return launch_chain_persistent(ch->ctx, ch->sets, ch->nsets, ch->nnodes, ch->nranks, ch->dtype, ch->count,
+                                       (cudaStream_t)stream);
+    if (!ch->exec) return NUNA_ERR_INVALID_ARG;
     if (cudaGraphLaunch(ch->exec, (cudaStream_t)stream) != cudaSuccess) return NUNA_ERR_CUDA;
     g_launches.fetch_add((unsigned long long)ch->nnodes, std::memory_order_relaxed);
     return NUNA_OK;

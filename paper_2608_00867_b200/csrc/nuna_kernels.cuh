@@ -325,6 +325,128 @@ k_oneshot_group(const RankPtrs p, const size_t count, const size_t ntiles)
     }
 }
 
+// ---- one-shot allreduce, co-located group staged through shared memory ---------------------------------
+//
+// The same logical group as above (one tile, every destination, on one compute unit), but the N
+// source slices of the tile are fetched ONCE per block by the bulk-copy engine: one elected thread
+// issues N one-dimensional cp.async.bulk copies global -> shared (plain form, this GPU's memory, no
+// multicast) that complete on an mbarrier; all N * tile bytes of a block are in flight at once without
+// holding a register.  Row d of the block (emulated rank d) then folds the N slices out of shared
+// memory in rank order and stores its destination.  Each emulated rank still reads all N sources and
+// does its own fold; what changes is where the N-fold re-read is served from (shared memory instead
+// of L1 / L2), so the L2 -> SM fabric carries every source byte once per tile.
+// One tile per block: the hardware block scheduler balances, and several resident blocks per SM
+// overlap one block's copy latency with another's fold.
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned arrivals)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(bar)), "r"(arrivals) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");   // visible to the bulk-copy engine
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+// Bulk copy of `bytes` (a multiple of 16; both addresses 16-byte aligned) from global to this block's shared memory.
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, unsigned bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity)
+{
+    unsigned done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait for phase `parity` of an mbarrier: after timeout_ns the thread latches NUNA_ERR_TIMEOUT in
+// *status and gives up (the caller skips its work and returns; nothing traps).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, unsigned* status, unsigned long long timeout_ns)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    unsigned polls = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++polls & 255u) == 0u && globaltimer_ns() - t0 > timeout_ns) {
+            atomicMax(status, 6u);                     // NUNA_ERR_TIMEOUT
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ uint4 ld_shared_v4(const uint4* p)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(p)));
+    return v;
+}
+
+__host__ __device__ constexpr int pow2_at_least(int n) { return n <= 1 ? 1 : n <= 2 ? 2 : n <= 4 ? 4 : n <= 8 ? 8 : 16; }
+
+// tv = vectors per source per tile (a multiple of kThreads / rows); shared memory = N * tv * 16 bytes.
+// (Filling the tile with ordinary 16-byte loads parked in shared memory instead of bulk copies was
+// measured too: never faster, and the registers that hold the loads in flight cost resident blocks.)
+template <int N, int DT>
+__global__ void __launch_bounds__(kThreads)
+k_oneshot_stage(const RankPtrs p, const size_t count, const unsigned tv, const int stream_stores,
+                unsigned* status, const unsigned long long timeout_ns)
+{
+    constexpr int kRows = pow2_at_least(N);
+    constexpr int kLanes = kThreads / kRows;
+    extern __shared__ __align__(128) unsigned char stage_raw[];
+    uint4* stage = reinterpret_cast<uint4*>(stage_raw);            // [N][tv]
+    __shared__ __align__(8) uint64_t bar;
+    const size_t nvec = count / Elem<DT>::kElems;
+    const size_t base = (size_t)blockIdx.x * tv;
+    const unsigned nv = base < nvec ? (unsigned)((nvec - base < tv) ? nvec - base : tv) : 0u;
+    if (threadIdx.x == 0) mbar_init(&bar, 1u);
+    __syncthreads();
+    pdl_wait();                                                     // before the first global access
+    if (nv != 0u) {
+        if (threadIdx.x == 0) {
+            mbar_expect_tx(&bar, (unsigned)N * nv * 16u);
+#pragma unroll
+            for (int r = 0; r < N; ++r) bulk_load(stage + (size_t)r * tv, p.src[r] + base, nv * 16u, &bar);
+        }
+        if (mbar_wait(&bar, 0u, status, timeout_ns)) {
+            const int d = threadIdx.x / kLanes;
+            if (d < N) {
+                uint4* out = p.dst[d] + base;
+                for (unsigned j = threadIdx.x % kLanes; j < nv; j += kLanes) {
+                    uint4 v[N];
+#pragma unroll
+                    for (int r = 0; r < N; ++r) v[r] = ld_shared_v4(stage + (size_t)r * tv + j);
+                    const uint4 o = fold_vectors<N, DT>(v);
+                    if (stream_stores) st_stream(out + j, o); else st_dst(out + j, o);
+                }
+            }
+        }
+    }
+    pdl_trigger();
+    const size_t tail0 = nvec * Elem<DT>::kElems;
+    if (tail0 < count) {
+        for (int d = blockIdx.x; d < N; d += gridDim.x) {
+            const size_t e = tail0 + threadIdx.x;
+            if (e < count) store_elem<DT>(p.dst[d], e, fold_scalar<N, DT>(p, e));
+        }
+    }
+}
+
 // ---- one-shot allreduce, a logical group per thread-block cluster --------------------------------------
 //
 // The hardware's own locality domain is the GPC: the blocks of a thread-block cluster are placed on
@@ -701,13 +823,6 @@ k_alltoall_scalar(const RankPtrs p, const int nranks, const size_t block)
 // `timeout_ns` the block latches NUNA_ERR_TIMEOUT in `status` and returns false;
 // the caller then skips the rest of its work and exits.  Nothing traps or hangs.
 
-__device__ __forceinline__ unsigned long long globaltimer_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
 __device__ __forceinline__ unsigned int ld_acquire(const unsigned int* p)
 {
     unsigned int v;
@@ -728,8 +843,6 @@ __device__ __forceinline__ bool flag_barrier(BarrierWords* bw, unsigned int expe
         asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(&bw->arrive) : "memory");
         if (prev == expected - 1) {
             bw->arrive = 0;                            // nobody touches it again before the epoch moves
-            bw->work[0] = 0;                           // everyone is past phase 1 and nobody is in phase 2 yet:
-            bw->work[1] = 0;                           // rewind both work cursors for this phase 2 / the next launch
             asm volatile("red.release.gpu.global.add.u32 [%0], 1;" :: "l"(&bw->epoch) : "memory");
         } else {
             const unsigned long long t0 = globaltimer_ns();
@@ -748,73 +861,145 @@ __device__ __forceinline__ bool flag_barrier(BarrierWords* bw, unsigned int expe
     return ok != 0;
 }
 
-// ---- fused two-shot allreduce ------------------------------------------------------------------------
+// ---- fused two-shot allreduce, synchronised by per-tile ready flags ---------------------------------------
 //
-// Persistent blocks (all co-resident; launched cooperatively).  Phase 1: emulated
-// rank r reduces chunk r of every source into shard scratch (a reduce-scatter
-// whose outputs live side by side in `scratch`).  Flag barrier.  Phase 2: put-style
-// allgather, chunk r is loaded once and stored into all N destinations.
-// chunk_vec = vectors per chunk; the last chunks may be short or empty.
-template <int N, int U, int DT>
-__global__ void __launch_bounds__(kThreads, min_blocks(N * U))
-k_twoshot_fused(const RankPtrs p, uint4* scratch, const size_t count, const size_t chunk_vec,
-                BarrierWords* bw, const unsigned long long timeout_ns)
+// Reduce-scatter, flag synchronisation and put-style allgather in ONE kernel, with no grid-wide barrier
+// and no host synchronisation.  The message is cut into tiles of tv vectors; the chunk a tile lies in
+// names the emulated rank that owns its reduction.  Every thread block takes ONE work item, numbered by a
+// ticket it draws from a device-wide counter when it starts; item i (0 <= i < tiles + lead) has two
+// halves, run side by side by the two halves of the block:
+//   produce tile i (while i < tiles; threads 0..127): the tile's N source slices are fetched into shared
+//       memory by bulk asynchronous copies (one thread issues them; they complete on an mbarrier), folded
+//       in rank order, stored to the shard scratch, and flag[i] = this launch's epoch is published with a
+//       release store (the producing rank's "chunk ready" signal);
+//   consume tile i - lead (once i >= lead; threads 128..255): acquire-poll that tile's flag until it
+//       holds this launch's epoch (bounded wait), then load the tile from the scratch once and store it
+//       into all N destinations (the put-style allgather).
+// `lead` is about what the whole device holds at once, so a tile is normally consumed long after it was
+// produced and its flag is found set; blocks flow from reducing into gathering without a common stop,
+// and because every block handles one item the hardware block scheduler does the load balancing.
+//
+// Progress: an item waits only for the flag of an item with a smaller ticket.  Tickets are drawn by
+// running blocks in the order they start, so that item belongs to a block that is running or has
+// finished, and whose own wait (if any) is again for a smaller ticket; by induction every wait ends, for
+// any grid size and without any co-residency requirement.  Every wait (flag, copy completion) is bounded
+// all the same: on expiry the block latches NUNA_ERR_TIMEOUT and leaves; nothing traps or spins forever.
+//
+// Replays: one 64-bit word in device memory carries the launch epoch (high half) and the next ticket (low
+// half), so a block learns both with its one atomic add.  The block that draws the last ticket knows that
+// every ticket of this launch is taken and stores (epoch + 1, 0) for the next launch.  Flags are compared
+// for equality with the epoch, so stale flags of earlier launches (or of another tiling) never match and
+// nothing is reset from the host.
+__device__ __forceinline__ void st_release(unsigned int* p, unsigned int v)
 {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+}
+
+// Polls *flag until it equals `want`.  Returns false (and latches the timeout) when timeout_ns runs out.
+__device__ __forceinline__ bool wait_flag(const unsigned int* flag, unsigned int want, unsigned long long timeout_ns,
+                                          unsigned int* status)
+{
+    if (ld_acquire(flag) == want) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    unsigned int polls = 0;
+    while (ld_acquire(flag) != want) {
+        if ((++polls & 63u) == 0u && globaltimer_ns() - t0 > timeout_ns) {
+            atomicMax(status, 6u);                     // NUNA_ERR_TIMEOUT
+            return false;
+        }
+    }
+    return true;
+}
+
+// Barrier among the 128 threads of one half of the block (ids 1 and 2; 0 is __syncthreads).
+__device__ __forceinline__ void half_sync(int id) { asm volatile("bar.sync %0, 128;" :: "r"(id) : "memory"); }
+
+// tv: vectors per tile; shared memory = N * tv * 16 bytes.  lead_max: upper bound of `lead`.
+// wait_bias: 0 in normal use; a test passes 1 so that consumers wait for a value nobody publishes.
+template <int N, int DT>
+__global__ void __launch_bounds__(kThreads)
+k_twoshot_flags(const RankPtrs p, uint4* scratch, unsigned int* flags, const size_t count, const unsigned tv,
+                const unsigned lead_max, BarrierWords* bw, const unsigned long long timeout_ns, const unsigned int wait_bias)
+{
+    constexpr unsigned kHalf = kThreads / 2;
+    extern __shared__ __align__(128) unsigned char stage_raw[];
+    uint4* stage = reinterpret_cast<uint4*>(stage_raw);            // [N][tv]
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ unsigned long long sh_ticket;
+    __shared__ int sh_ok, sh_landed;
     const size_t nvec = count / Elem<DT>::kElems;
-    const size_t tiles_per_chunk = (chunk_vec + kThreads * U - 1) / (kThreads * U);
-    const size_t nitems = tiles_per_chunk * N;
-    __shared__ unsigned sh_item;
-    unsigned int epoch0 = 0;
-    if (threadIdx.x == 0) epoch0 = ld_acquire(&bw->epoch);
-
-    // Work distribution inside the persistent grid: a block's first item is its own index (no latency
-    // at start), every further item is claimed from a device-wide cursor, the next claim being issued
-    // before the current item is processed.  Static striding left the blocks of the die with more SMs
-    // behind (its SMs share the same memory bandwidth among more blocks); claiming evens that out.
-    auto for_each_item = [&](unsigned int* cursor, auto&& body) {
-        size_t item = blockIdx.x;
-        unsigned next = 0;
-        while (item < nitems) {
-            if (threadIdx.x == 0) next = atomicAdd(cursor, 1u);
-            body(item);
-            if (threadIdx.x == 0) sh_item = next;
-            __syncthreads();
-            item = (size_t)gridDim.x + sh_item;
-            __syncthreads();
-        }
-    };
-
-    for_each_item(&bw->work[0], [&](size_t item) {
-        const int r = (int)(item % N);                 // rank fastest: neighbouring blocks work on different chunks
-        const size_t tile = item / N;
-        const size_t off = (size_t)r * chunk_vec;
-        if (off >= nvec) return;
-        const size_t len = (nvec - off < chunk_vec) ? nvec - off : chunk_vec;
-        reduce_tile<N, U, DT, false>(p, scratch + off, off, len, tile);
-    });
-    const size_t tail0 = nvec * Elem<DT>::kElems;             // ragged tail: reduced by block 0 into scratch
-    if (tail0 < count && blockIdx.x == 0) {
-        const size_t e = tail0 + threadIdx.x;
-        if (e < count) store_elem<DT>(scratch, e, fold_scalar<N, DT>(p, e));
+    const size_t tail0 = nvec * Elem<DT>::kElems;
+    const size_t ntiles = nvec ? (nvec + tv - 1) / tv : 1;         // a ragged tail rides on the last tile
+    const size_t lead = ntiles < lead_max ? ntiles : lead_max;
+    if (threadIdx.x == 0) mbar_init(&bar, 1u);
+    pdl_wait();                                                     // before the first global access
+    if (threadIdx.x == 0) {
+        const unsigned long long t = atomicAdd(&bw->ticket, 1ull);  // epoch and ticket in one round trip
+        if ((unsigned)t == gridDim.x - 1u)                          // the last ticket: set up the next launch
+            *reinterpret_cast<volatile unsigned long long*>(&bw->ticket) = ((t >> 32) + 1ull) << 32;
+        sh_ticket = t;
     }
+    __syncthreads();
+    const size_t item = (unsigned)sh_ticket;
+    const unsigned epoch1 = (unsigned)(sh_ticket >> 32) + 1u;
+    const bool produce = item < ntiles, consume = item >= lead && item < ntiles + lead;
 
-    if (!flag_barrier(bw, gridDim.x, epoch0, timeout_ns)) return;
-
-    for_each_item(&bw->work[1], [&](size_t item) {
-        const int r = (int)(item % N);
-        const size_t tile = item / N;
-        const size_t off = (size_t)r * chunk_vec;
-        if (off >= nvec) return;
-        const size_t len = (nvec - off < chunk_vec) ? nvec - off : chunk_vec;
-        gather_tile<U>(scratch + off, p, 0, N, off, len, tile, true);
-    });
-    if (tail0 < count && blockIdx.x == 0) {
-        const size_t e = tail0 + threadIdx.x;
-        if (e < count) {
-            const uint32_t v = load_elem_cg<DT>(scratch, e);
-            for (int d = 0; d < N; ++d) store_elem<DT>(p.dst[d], e, v);
+    if (threadIdx.x < kHalf) {
+        // ---- produce half ----
+        if (produce) {
+            const size_t pbase = item * tv;
+            const unsigned pnv = pbase < nvec ? (unsigned)((nvec - pbase < tv) ? nvec - pbase : tv) : 0u;
+            bool landed = true;
+            if (pnv != 0u) {
+                if (threadIdx.x == 0) {
+                    mbar_expect_tx(&bar, (unsigned)N * pnv * 16u);
+#pragma unroll
+                    for (int r = 0; r < N; ++r) bulk_load(stage + (size_t)r * tv, p.src[r] + pbase, pnv * 16u, &bar);
+                }
+                landed = mbar_wait(&bar, 0u, &bw->status, timeout_ns);
+                if (landed) {
+                    for (unsigned j = threadIdx.x; j < pnv; j += kHalf) {
+                        uint4 v[N];
+#pragma unroll
+                        for (int r = 0; r < N; ++r) v[r] = ld_shared_v4(stage + (size_t)r * tv + j);
+                        st_dst(scratch + pbase + j, fold_vectors<N, DT>(v));
+                    }
+                }
+            }
+            if (item == ntiles - 1 && tail0 < count) {
+                const size_t e = tail0 + threadIdx.x;
+                if (e < count) store_elem<DT>(scratch, e, fold_scalar<N, DT>(p, e));
+            }
+            if (threadIdx.x == 0) sh_landed = 1;
+            half_sync(1);
+            if (!landed) sh_landed = 0;
+            half_sync(1);                              // every thread's shard stores are issued ...
+            if (threadIdx.x == 0 && sh_landed) st_release(flags + item, epoch1);   // ... and ordered before the flag
+        }
+    } else {
+        // ---- consume half ----
+        if (consume) {
+            const size_t ct = item - lead, cbase = ct * tv;
+            if (threadIdx.x == kHalf) sh_ok = wait_flag(flags + ct, epoch1 + wait_bias, timeout_ns, &bw->status) ? 1 : 0;
+            half_sync(2);                              // flag acquired by one thread -> every thread may read the tile
+            if (sh_ok) {
+                const unsigned cnv = cbase < nvec ? (unsigned)((nvec - cbase < tv) ? nvec - cbase : tv) : 0u;
+                for (unsigned j = threadIdx.x - kHalf; j < cnv; j += kHalf) {
+                    const uint4 c = ld_cg(scratch + cbase + j);
+#pragma unroll
+                    for (int d = 0; d < N; ++d) st_stream(p.dst[d] + cbase + j, c);
+                }
+                if (ct == ntiles - 1 && tail0 < count) {
+                    const size_t e = tail0 + (threadIdx.x - kHalf);
+                    if (e < count) {
+                        const uint32_t w = load_elem_cg<DT>(scratch, e);
+                        for (int d = 0; d < N; ++d) store_elem<DT>(p.dst[d], e, w);
+                    }
+                }
+            }
         }
     }
+    pdl_trigger();
 }
 
 // Two-shot without the intermediate: the block that reduces a tile stores it into all N destinations.
@@ -853,6 +1038,90 @@ k_twoshot_put(const RankPtrs p, const size_t count, const size_t ntiles)
             const uint32_t v = fold_scalar<N, DT>(p, e);
             for (int d = 0; d < N; ++d) store_elem<DT>(p.dst[d], e, v);
         }
+    }
+}
+
+// ---- decode-step chain in one kernel --------------------------------------------------------------------
+//
+// For small nodes a kernel launch (about 1.1 us even as a graph node with dependent launch) costs many
+// times the data time, so the whole chain of back-to-back one-shot allreduces runs as ONE kernel on one
+// thread-block cluster.  Node k works on buffer set k mod nsets; the node boundary is a cluster barrier
+// with release / acquire semantics, so node k+1 reads only after every block has finished writing node k
+// (a node may read what its predecessor wrote).  Within a node the work is the co-located one-shot:
+// block b takes tiles b, b + blocks, ...; row d of a block is emulated rank d's item for that tile.
+// Loads are ordinary coherent global loads (a source may have been written by the previous node).
+__device__ __forceinline__ unsigned cluster_nctarank()
+{
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+
+__device__ __forceinline__ uint4 ld_coherent(const uint4* p)
+{
+    uint4 v;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+
+template <int N, int DT>
+__global__ void __launch_bounds__(kThreads, 1)
+k_chain_persistent(const __grid_constant__ ChainSets sets, const int nsets, const int nnodes, const size_t count)
+{
+    constexpr int C = pow2_at_least(N) > 8 ? 8 : pow2_at_least(N);
+    constexpr int kLanes = kThreads / C;
+    constexpr int kSplit = (N + C - 1) / C;
+    const unsigned nblk = cluster_nctarank(), blk = cluster_ctarank();
+    const size_t nvec = count / Elem<DT>::kElems;
+    const size_t nitems = ((nvec + kLanes - 1) / kLanes) * kSplit;
+    const size_t tail0 = nvec * Elem<DT>::kElems;
+    const int row = threadIdx.x / kLanes, lane = threadIdx.x % kLanes;
+    int set = 0;
+    for (int node = 0; node < nnodes; ++node) {
+        const RankPtrs& p = sets.s[set];
+        // two items per step so that 2N loads are in flight per thread
+        for (size_t it = blk; it < nitems; it += 2 * (size_t)nblk) {
+            uint4 v[2][N];
+            size_t vi[2];
+            int dd[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const size_t item = it + (size_t)h * nblk;
+                dd[h] = (int)(item % kSplit) * C + row;
+                vi[h] = (item / kSplit) * kLanes + lane;
+                if (item < nitems && dd[h] < N && vi[h] < nvec) {
+#pragma unroll
+                    for (int r = 0; r < N; ++r) v[h][r] = ld_coherent(p.src[r] + vi[h]);
+                } else {
+                    dd[h] = -1;
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+                if (dd[h] >= 0) st_dst(p.dst[dd[h]] + vi[h], fold_vectors<N, DT>(v[h]));
+        }
+        if (tail0 < count && blk == 0) {
+            const size_t e = tail0 + lane;
+            for (int d = row; d < N && e < count; d += C) {
+                uint32_t w;
+                if (DT == kF32) {
+                    float acc = __uint_as_float(*reinterpret_cast<const volatile uint32_t*>(reinterpret_cast<const uint32_t*>(p.src[0]) + e));
+                    for (int r = 1; r < N; ++r)
+                        acc = __fadd_rn(acc, __uint_as_float(*reinterpret_cast<const volatile uint32_t*>(reinterpret_cast<const uint32_t*>(p.src[r]) + e)));
+                    w = __float_as_uint(acc);
+                } else {
+                    float acc, unused;
+                    widen_word<DT>(acc, unused, (uint32_t)*reinterpret_cast<const volatile uint16_t*>(reinterpret_cast<const uint16_t*>(p.src[0]) + e));
+                    for (int r = 1; r < N; ++r)
+                        acc = add_narrow<DT>(acc, *reinterpret_cast<const volatile uint16_t*>(reinterpret_cast<const uint16_t*>(p.src[r]) + e));
+                    w = pack2<DT>(acc, 0.0f) & 0xFFFFu;
+                }
+                store_elem<DT>(p.dst[d], e, w);
+            }
+        }
+        cluster_sync();                                // node boundary: writes of node k before reads of node k+1
+        set = (set + 1 == nsets) ? 0 : set + 1;
     }
 }
 

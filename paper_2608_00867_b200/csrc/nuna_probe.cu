@@ -20,6 +20,7 @@
 // The sampled words are saved before and restored after the measurement, so buffer contents are
 // unchanged on return.  Not capturable: it allocates, copies and synchronises.
 #include "nuna_internal.h"
+#include "nuna_debug.h"
 
 #include <algorithm>
 #include <cmath>

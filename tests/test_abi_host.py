@@ -18,14 +18,23 @@ def built_library():
 
 
 def declared_functions():
+    """Functions declared by the public header(s) and by the internal header of the test hooks."""
+    headers = [os.path.join(ROOT, "include", fn) for fn in os.listdir(os.path.join(ROOT, "include")) if fn.endswith(".h")]
+    headers.append(os.path.join(ROOT, "paper_2608_00867_b200", "csrc", "nuna_debug.h"))
     names = set()
-    for fn in os.listdir(os.path.join(ROOT, "include")):
-        if not fn.endswith(".h"):
-            continue
-        text = open(os.path.join(ROOT, "include", fn)).read()
+    for path in headers:
+        text = open(path).read()
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
         names |= set(re.findall(r"\b(nuna_[a-z0-9_]+)\s*\(", text))
     return sorted(names)
+
+
+def test_no_undeclared_exports():
+    """Every nuna_* symbol the library exports is declared in the public header or in the debug header."""
+    import subprocess
+    out = subprocess.run(["nm", "-D", "--defined-only", nb._LIB_PATH], capture_output=True, text=True, check=True).stdout
+    exported = {ln.split()[-1] for ln in out.splitlines() if ln.split() and ln.split()[-1].startswith("nuna_")}
+    assert exported <= set(declared_functions()), exported - set(declared_functions())
 
 
 def test_every_declared_symbol_is_exported():
@@ -55,7 +64,8 @@ def test_validation_happens_before_any_cuda_call():
     assert call(ok_src, [A + 8192, A + 8192 + 16], 5, dtype=nb.NUNA_BF16) in (nb.NUNA_ERR_CUDA, nb.NUNA_OK)  # 10 bytes: fine
     assert call(ok_src, ok_dst, 8, dtype=77) == nb.NUNA_ERR_UNSUPPORTED_DTYPE
     assert call(ok_src, ok_dst, 8, flags=3) == nb.NUNA_ERR_INVALID_ARG
-    assert call(ok_src, ok_dst, 8, flags=1 << 9) == nb.NUNA_ERR_INVALID_ARG
+    assert call(ok_src, ok_dst, 8, flags=1 << 13) == nb.NUNA_ERR_INVALID_ARG
+    assert call(ok_src, ok_dst, 8, flags=nb.NUNA_CHAIN_PERSISTENT) == nb.NUNA_ERR_INVALID_ARG    # chain-only bit
     assert call(ok_src, [A + 8192, 0], 8) == nb.NUNA_ERR_INVALID_ARG
     assert call(ok_src, [A + 8192, A + 12288 + 2], 8) == nb.NUNA_ERR_ALIGNMENT
     assert call(ok_src, [A + 8192, A + 8192 + 16], 9) == nb.NUNA_ERR_ALIAS     # 18 bytes each: overlap

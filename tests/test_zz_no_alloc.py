@@ -4,14 +4,15 @@ Some users of this library cannot allocate device memory where they call it: a s
 process whose framework owns every byte of the GPU through its own pool, or a request loop
 that must not pay for (or survive the failure of) a cudaMalloc.  For them the library has one
 entry point whose scratch is a fixed array compiled into it.  This file checks that entry
-point, through the C ABI, against the ordinary two-shot allreduce: same bits, twice in a row
-(the array keeps the first call's shard, which must not leak into the second result), and a
-clear refusal beyond the array's size.  It is collected last on purpose.
+point, through the C ABI, against the ordinary two-shot allreduce and against the CPU oracle:
+same bits, twice in a row (the array keeps the first call's shard, which must not leak into the
+second result), and a clear refusal beyond the array's size.  It is collected last on purpose.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2608_00867_b200 import binding as nb
 from paper_2608_00867_b200 import workloads
 
@@ -41,8 +42,13 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point():
     second = workloads.special_values(5, 100003, seed=2)
     for src, count in ((first, w.count), (second, 100003)):
         ref, got = run_both(src, count)
+        want = oracle.allreduce(src, nthreads=4)[0]
+        nan = ((want & 0x7F80) == 0x7F80) & ((want & 0x007F) != 0)
         for r, g in zip(ref, got):
             assert torch.equal(r, g)                            # bit for bit, every destination
+            h = g.cpu().numpy().view(np.uint16)
+            assert np.array_equal(h[~nan], want[~nan])          # and the same bits as the CPU oracle
+            assert (((h[nan] & 0x7F80) == 0x7F80) & ((h[nan] & 0x007F) != 0)).all()
     # and once more with the first message: the array now holds the second call's shard
     ref, got = run_both(first, w.count)
     assert all(torch.equal(r, g) for r, g in zip(ref, got))
@@ -63,3 +69,26 @@ def test_sizes_beyond_the_fixed_array_are_refused():
     src = workloads.rank_buffers(n, count, "normal", seed=8)
     ref, got = run_both(src, count)
     assert all(torch.equal(r, g) for r, g in zip(ref, got))
+    assert np.array_equal(got[0].cpu().numpy().view(np.uint16), oracle.allreduce(src, nthreads=4)[0])
+    assert nb.nuna_device_status() == nb.NUNA_OK                # also reads the fixed arrays' own status word
+
+
+@pytest.mark.parametrize("dtype", ["f16", "f32"])
+def test_other_element_types_and_the_limit_in_bytes(dtype):
+    """The limit is the array's size in bytes: 2 Mi 16-bit elements, 1 Mi binary32 elements."""
+    n = 3
+    code = nb.DTYPE_BY_NAME[dtype]
+    tdt = torch.int32 if dtype == "f32" else torch.int16
+    limit = nb.NUNA_STATIC_MAX_COUNT * 2 // nb.ELEM_SIZE[code]
+    src = workloads.rank_buffers_typed(n, limit, "normal", 17, dtype)
+    want = oracle.allreduce(src, nthreads=4, dtype=dtype)[0]
+    dsrc = [torch.from_numpy(a.view(np.int32 if dtype == "f32" else np.int16).copy()).cuda() for a in src]
+    for _ in range(2):                                          # two calls in a row on the shared array
+        dst = [torch.zeros(limit, dtype=tdt, device="cuda") for _ in range(n)]
+        nb.nuna_allreduce_twoshot_static(dsrc, dst, limit, dtype=code)
+        torch.cuda.synchronize()
+        for d in dst:
+            assert np.array_equal(d.cpu().numpy().view(want.dtype), want)
+    over = limit + 16 // nb.ELEM_SIZE[code]
+    big = [torch.zeros(over, dtype=tdt, device="cuda") for _ in range(2 * n)]
+    assert nb.nuna_allreduce_twoshot_static(big[:n], big[n:], over, dtype=code, check=False) == nb.NUNA_ERR_TOO_LARGE
