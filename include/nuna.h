@@ -83,10 +83,8 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 #define NUNA_HINT_RESIDENT    32u
 /* `flags`, bit 6: launch with programmatic stream serialization.  The kernel may be scheduled while its
  * predecessor in the stream drains; it waits for that grid's completion and memory visibility before
- * its first global access, so results are those of an ordinary stream-ordered launch.  The flag-
- * synchronised two-shot is launched cooperatively without this flag and as an ordinary (non-cooperative)
- * launch with it; the round-robin one-shot ignores it above 16 MiB of sources, where it was measured
- * not to pay.                                                                                           */
+ * its first global access, so results are those of an ordinary stream-ordered launch.  The round-robin
+ * one-shot ignores it above 16 MiB of sources, where it was measured not to pay.                         */
 #define NUNA_LAUNCH_PDL       64u
 /* `flags`, bit 7, with NUNA_PLACE_AWARE on nuna_allreduce_oneshot: dispatch the co-located groups through
  * per-SM work lists.  The lists are planned by Algorithm 1 from the topology the last
@@ -112,10 +110,17 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 /* `flags`, bits 11-12, nuna_chain_create only: run the chain as ONE kernel on a single thread-block
  * cluster with a cluster barrier as node boundary (NUNA_CHAIN_PERSISTENT; one-shot nodes, at most 8
  * buffer sets, at most 4 MiB per rank, else NUNA_ERR_INVALID_ARG), or always as a CUDA graph of one kernel
- * per node (NUNA_CHAIN_GRAPH).  With neither bit the library picks the single kernel for small nodes
- * (up to 128 KiB per rank), where a launch per node costs more than the node's data movement.           */
+ * per node (NUNA_CHAIN_GRAPH).  With neither bit the library picks by measurement, which on B200 means the
+ * graph at every size: the single kernel's node (two dependent memory round trips on one cluster's SMs)
+ * costs 1.27 us at 16 KiB per rank against 1.15 us for a graph node launched behind its predecessor.    */
 #define NUNA_CHAIN_PERSISTENT 2048u
 #define NUNA_CHAIN_GRAPH      4096u
+/* `flags`, bit 13, flag-synchronised two-shot only: publish and poll the ready flags with system-scope
+ * release / acquire (st.release.sys / ld.acquire.sys) instead of device scope.  On one GPU the result and
+ * the algorithm are the same; this is the form the synchronisation takes when the rank buffers, the shard
+ * and the flags live in peer GPUs' memory (plain loads and stores through peer-mapped pointers).  Not tested
+ * across GPUs.                                                                                          */
+#define NUNA_TWOSHOT_SYS_SCOPE 8192u
 
 /* ---- topology probe --------------------------------------------------------------------------------
  * Result of nuna_probe_topology: caller-owned, plain data, fixed maximum sizes.  Latencies are in SM
@@ -129,6 +134,10 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 #define NUNA_HIST_BINS        48
 #define NUNA_HIST_FIRST       200
 #define NUNA_HIST_STEP        4
+#define NUNA_SCAN_LINES       512   /* consecutive 128-byte lines of buffer 0 whose home domain is mapped      */
+#define NUNA_SCAN_RUN_BINS    16    /* run-length histogram: bin i = runs of i+1 lines, last bin = that or more */
+#define NUNA_SCAN_LEVELS      3     /* granularities of the home-share table: 4 KiB, 64 KiB, 2 MiB             */
+#define NUNA_SCAN_BLOCKS      8     /* consecutive blocks of each granularity, from the start of buffer 0       */
 
 typedef struct nuna_topology {
     int num_sms;                     /* cudaDeviceProp.multiProcessorCount                                 */
@@ -161,14 +170,30 @@ typedef struct nuna_topology {
      * (Section 6.2).                                                                                     */
     unsigned hist_near[NUNA_HIST_BINS];
     unsigned hist_far[NUNA_HIST_BINS];
+    /* At which granularity does the home domain of an address change (Section 3.2: latency depends on the
+     * target address)?  scan_home[i] is the home domain of the i-th of scan_lines CONSECUTIVE 128-byte
+     * lines of buffer 0 (from its first 128-byte boundary); scan_run_hist counts the runs of equal home
+     * among them by length, scan_longest_run is the longest.  scan_level_share[g][b] is the share of 16
+     * sampled lines at home in domain 0 inside the b-th consecutive block of 4 KiB (g = 0), 64 KiB (1) or
+     * 2 MiB (2) of buffer 0, -1 where buffer 0 is too short; scan_level_spread[g] = max - min over the
+     * blocks of that granularity (-1 with fewer than two blocks).  A spread near zero with shares near one
+     * half means the address hash is finer than that granularity: no block of that size is "near" a domain.
+     * All zero / -1 when the verdict is uniform.                                                          */
+    int scan_lines;
+    int scan_longest_run;
+    unsigned char scan_home[NUNA_SCAN_LINES];
+    unsigned scan_run_hist[NUNA_SCAN_RUN_BINS];
+    float scan_level_share[NUNA_SCAN_LEVELS][NUNA_SCAN_BLOCKS];
+    float scan_level_spread[NUNA_SCAN_LEVELS];
 } nuna_topology_t;
 
 /* Measures, for every SM (indexed by %smid) and every buffer, the latency of dependent L2-only loads
  * to sampled lines of the caller's buffers (the analogue of the paper's per-compute-unit, per-address
  * remote-access sweep, Section 3.2), plus each SM's cold DRAM latency, clusters the SMs into domains
+ * maps the home domain of a window of consecutive lines and of blocks of 4 KiB / 64 KiB / 2 MiB of buffer 0,
  * and stores the result in *out and in the device context (where NUNA_PLACE_SM_LISTS plans read it).
  * bufs: HOST array of nbufs (<= NUNA_MAX_PROBE_BUFS) device pointers, bytes[b] >= 128 each, 16-byte
- * aligned.  One 8-byte word per sampled line is overwritten during the measurement and restored
+ * aligned.  One 8-byte word per sampled line (about 3000 lines at most) is overwritten during the measurement and restored
  * before return; the buffers must not be in use by other work meanwhile.  Synchronises `stream`,
  * allocates temporary device memory (about 2.3 x the L2 size): NUNA_ERR_CAPTURING on a capturing
  * stream.  Work lists planned earlier for NUNA_PLACE_SM_LISTS are retired and rebuilt under the new
@@ -240,14 +265,17 @@ int nuna_allreduce_oneshot(const void* const* src, void* const* dst, int nranks,
 
 /* Two-shot allreduce: reduce-scatter over N contiguous chunks (the chunk a tile lies in names the emulated
  * rank that reduces it), per-tile ready flags in place of a host synchronisation, then a put-style
- * allgather of the reduced tiles into every destination -- all in one kernel of co-resident thread
- * blocks.  A block that has reduced a tile publishes the tile's flag with a release store; the block that
- * gathers the tile acquire-polls that flag (bounded wait: on expiry NUNA_ERR_TIMEOUT is latched and the
- * block returns).  Same bits as the one-shot.  Any `count`; chunk = ceil(count/N) rounded up to a whole
- * 16-byte vector, trailing chunks may be short or empty.  Uses the context's shard scratch (count*elemsize
- * bytes plus one flag word per 4 KiB, grown on demand; an outgrown scratch stays allocated until
- * nuna_shutdown because captured graphs may still name it) unless NUNA_TWOSHOT_PUT is set.  Calls that
- * share the context must be stream-ordered with respect to each other.                                 */
+ * allgather of the reduced tiles into every destination -- all in one kernel.  Every thread block takes one
+ * work item, numbered by a ticket drawn from a device counter: it reduces one tile into the shard scratch
+ * and publishes the tile's flag with a release store, and it gathers an earlier tile into all destinations
+ * after acquire-polling that tile's flag (bounded wait: on expiry NUNA_ERR_TIMEOUT is latched and the block
+ * returns).  A wait is only ever for an item with a smaller ticket, held by a block that already runs, so
+ * the kernel needs no co-residency guarantee and no cooperative launch.  Consumed shard lines are dropped
+ * from L2 (discard) instead of being written back.  Same bits as the one-shot.  Any `count`; chunk =
+ * ceil(count/N) rounded up to a whole 16-byte vector, trailing chunks may be short or empty.  Uses the
+ * context's shard scratch (count*elemsize bytes plus one flag word per 256 bytes, grown on demand; an
+ * outgrown scratch stays allocated until nuna_shutdown because captured graphs may still name it) unless
+ * NUNA_TWOSHOT_PUT is set.  Calls that share the context must be stream-ordered with respect to each other. */
 int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
                            size_t count, int dtype, unsigned flags, void* stream);
 
@@ -316,9 +344,9 @@ int nuna_allreduce_host(const void* const* src, void* const* dst, int nranks,
  * device pointers, set s occupying entries [s*nranks, (s+1)*nranks); node k works on set k mod nsets
  * and starts reading only after node k-1 has finished writing.  flags as for the allreduce calls
  * (NUNA_LAUNCH_PDL overlaps each node's launch with its predecessor's drain); two_shot selects
- * nuna_allreduce_twoshot.  Small one-shot nodes run as a single kernel instead of a graph (see
+ * nuna_allreduce_twoshot.  One-shot nodes can also run as a single kernel instead of a graph (see
  * NUNA_CHAIN_PERSISTENT / NUNA_CHAIN_GRAPH): one thread-block cluster loops over the nodes with a cluster
- * barrier between them, which removes the per-node launch cost.  Creation allocates and synchronises
+ * barrier between them, which removes the per-node launch.  Creation allocates and synchronises
  * nothing on the caller's streams; the chain reads the buffers named at creation on every launch.
  * *chain_out is an opaque handle.                                                                       */
 int nuna_chain_create(const void* const* src_sets, void* const* dst_sets, int nsets, int nnodes, int nranks,

@@ -34,10 +34,12 @@ NUNA_PLACE_STAGED = 512
 NUNA_TWOSHOT_SYNC = 1024
 NUNA_CHAIN_PERSISTENT = 2048
 NUNA_CHAIN_GRAPH = 4096
+NUNA_TWOSHOT_SYS_SCOPE = 8192
 
 NUNA_MAX_SMS, NUNA_MAX_PROBE_BUFS, NUNA_PROBE_REGIONS, NUNA_MAX_PROBE_LINES = 256, 32, 8, 2048
 NUNA_TOPO_UNIFORM, NUNA_TOPO_NONUNIFORM = 0, 1
 NUNA_HIST_BINS, NUNA_HIST_FIRST, NUNA_HIST_STEP = 48, 200, 4
+NUNA_SCAN_LINES, NUNA_SCAN_RUN_BINS, NUNA_SCAN_LEVELS, NUNA_SCAN_BLOCKS = 512, 16, 3, 8
 NUNA_OPT_BLOCKS, NUNA_OPT_UNROLL, NUNA_OPT_COLOC, NUNA_OPT_AUTO_MIN_BYTES, NUNA_OPT_TIMEOUT_MS = 0, 1, 2, 3, 4
 NUNA_OPT_DOMAINS, NUNA_OPT_STAGE_VECS, NUNA_OPT_TWOSHOT_VECS = 5, 6, 7
 
@@ -63,6 +65,11 @@ class NunaTopology(ctypes.Structure):
         ("line_home", ctypes.c_ubyte * NUNA_MAX_PROBE_LINES),
         ("hist_near", ctypes.c_uint * NUNA_HIST_BINS),
         ("hist_far", ctypes.c_uint * NUNA_HIST_BINS),
+        ("scan_lines", ctypes.c_int), ("scan_longest_run", ctypes.c_int),
+        ("scan_home", ctypes.c_ubyte * NUNA_SCAN_LINES),
+        ("scan_run_hist", ctypes.c_uint * NUNA_SCAN_RUN_BINS),
+        ("scan_level_share", (ctypes.c_float * NUNA_SCAN_BLOCKS) * NUNA_SCAN_LEVELS),
+        ("scan_level_spread", ctypes.c_float * NUNA_SCAN_LEVELS),
     ]
 
 
@@ -145,8 +152,10 @@ def lib() -> ctypes.CDLL:
         L.nuna_shutdown.restype = ctypes.c_int
         L.nuna_debug_barrier_selftest.argtypes = [ctypes.c_uint, ctypes.c_uint, ctypes.c_uint, ctypes.POINTER(ctypes.c_uint)]
         L.nuna_debug_barrier_selftest.restype = ctypes.c_int
-        L.nuna_debug_twoshot_unset_flags.argtypes = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint]
-        L.nuna_debug_twoshot_unset_flags.restype = ctypes.c_int
+        L.nuna_debug_access_latency.argtypes = [vpp, vpp, ctypes.c_size_t, ctypes.c_int, ctypes.POINTER(ctypes.c_uint)]
+        L.nuna_debug_access_latency.restype = ctypes.c_int
+        L.nuna_debug_twoshot.argtypes = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint, ctypes.c_uint]
+        L.nuna_debug_twoshot.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -368,9 +377,27 @@ def nuna_shutdown() -> int:
     return lib().nuna_shutdown()
 
 
-def debug_twoshot_unset_flags(src, dst, count, dtype=NUNA_BF16, timeout_ms: int = 50) -> int:
-    """Test hook: a two-shot whose consumers wait for ready flags that nobody publishes (bounded waits)."""
-    return lib().nuna_debug_twoshot_unset_flags(ptr_table(src), ptr_table(dst), len(src), count, dtype, timeout_ms)
+DEBUG_LAT_BINS, DEBUG_LAT_STEP = 64, 32
+
+
+def debug_access_latency(src, dst, count, placement: int, launches: int = 1):
+    """Histogram (numpy uint32[DEBUG_LAT_BINS], bins of DEBUG_LAT_STEP cycles) of first-load latencies of the
+    8-rank bf16 one-shot under a placement: 0 round-robin, 1 co-located groups, 2 per-SM work lists."""
+    import numpy as np
+    hist = np.zeros(DEBUG_LAT_BINS, dtype=np.uint32)
+    for _ in range(launches):
+        st = lib().nuna_debug_access_latency(ptr_table(src), ptr_table(dst), count, placement,
+                                             hist.ctypes.data_as(ctypes.POINTER(ctypes.c_uint)))
+        if st != NUNA_OK:
+            raise NunaError(st, "nuna_debug_access_latency")
+    return hist
+
+
+def debug_twoshot(src, dst, count, dtype=NUNA_BF16, timeout_ms: int = 1000, unset_flags: bool = False) -> int:
+    """Test hook: the flag-synchronised two-shot with an explicit timeout; with unset_flags its consumers
+    wait for flags nobody publishes, so every (bounded) wait runs out."""
+    return lib().nuna_debug_twoshot(ptr_table(src), ptr_table(dst), len(src), count, dtype, timeout_ms,
+                                    1 if unset_flags else 0)
 
 
 def debug_barrier_selftest(grid: int, expected: int, timeout_ms: int):

@@ -67,6 +67,7 @@ int get_context(Context** out)
         c->opt.domains = env_int("NUNA_DOMAINS", 0);
         c->opt.stage_vecs = env_int("NUNA_STAGE_VECS", 0);
         c->opt.twoshot_vecs = env_int("NUNA_TWOSHOT_VECS", 0);
+        c->opt.keep_shard = env_int("NUNA_KEEP_SHARD", 0);
         g_ctx[dev] = c;
     }
     *out = g_ctx[dev];
@@ -113,7 +114,8 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
     if (nranks < 1) return NUNA_ERR_INVALID_ARG;
     if (dtype != NUNA_BF16 && dtype != NUNA_F16 && dtype != NUNA_F32) return NUNA_ERR_UNSUPPORTED_DTYPE;
     if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT | NUNA_HINT_RESIDENT | NUNA_LAUNCH_PDL | NUNA_PLACE_SM_LISTS |
-                   NUNA_PLACE_CLUSTER | NUNA_PLACE_STAGED | NUNA_TWOSHOT_SYNC | NUNA_CHAIN_PERSISTENT | NUNA_CHAIN_GRAPH)) != 0u ||
+                   NUNA_PLACE_CLUSTER | NUNA_PLACE_STAGED | NUNA_TWOSHOT_SYNC | NUNA_CHAIN_PERSISTENT | NUNA_CHAIN_GRAPH |
+                   NUNA_TWOSHOT_SYS_SCOPE)) != 0u ||
         (flags & NUNA_PLACE_MASK) == 3u)
         return NUNA_ERR_INVALID_ARG;
     if (src_elems > ((size_t)1 << 40) || dst_elems > ((size_t)1 << 40)) return NUNA_ERR_TOO_LARGE;
@@ -466,7 +468,7 @@ int prepare_oneshot(Context* c, int nranks, int dtype, size_t count, unsigned fl
 template <int N, int C, int DT>
 static int launch_sm_lists(Context* c, const Options& o, const RankPtrs& p, size_t count, unsigned mode, cudaStream_t stream)
 {
-    auto k = k_oneshot_sm<N, C, DT>;
+    auto k = k_oneshot_sm<N, C, DT, false>;
     SmPlan pl;
     const int st = get_sm_plan(c, N, count / Elem<DT>::kElems, C, o.domains, stream, &pl);
     if (st != NUNA_OK) return st;
@@ -476,7 +478,7 @@ static int launch_sm_lists(Context* c, const Options& o, const RankPtrs& p, size
     const size_t cap = (size_t)c->num_sms * (size_t)NUNA_OCC(k);
     const unsigned grid = (unsigned)std::min(cap, std::max<size_t>((size_t)c->num_sms, (size_t)pl.total));
     const unsigned blocks_per_sm = (unsigned)std::max<size_t>(1, grid / (size_t)c->num_sms);
-    return launch(k, grid, stream, mode, p, count, sl, blocks_per_sm);
+    return launch(k, grid, stream, mode, p, count, sl, blocks_per_sm, (unsigned*)nullptr);
 }
 
 template <int N, int DT>
@@ -584,7 +586,7 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
 // tv = 0 picks the tile size by message size.  min_tv is the smallest tile the flag array was sized for.
 int launch_twoshot_flags(int num_sms, int blocks_override, const RankPtrs& p, int nranks, int dtype, size_t count,
                          unsigned tv, unsigned min_tv, uint4* scratch, unsigned* tile_flags, BarrierWords* bw,
-                         unsigned long long timeout_ns, bool pdl, unsigned wait_bias, cudaStream_t stream)
+                         unsigned long long timeout_ns, bool pdl, unsigned debug_bits, cudaStream_t stream)
 {
     const size_t bytes = count * elem_size(dtype);
     const size_t nvec = count / elems_per_vec(dtype);
@@ -606,10 +608,12 @@ int launch_twoshot_flags(int num_sms, int blocks_override, const RankPtrs& p, in
     const unsigned grid = (unsigned)(ntiles + lead);
     return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
         constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
-        auto k = k_twoshot_flags<N, DT>;
         t_dyn_smem = (unsigned)N * tv * 16u;
-        return launch(k, grid, stream, pdl ? kLaunchPdl : kLaunchPlain, p, scratch, tile_flags, count, tv, lead_max, bw,
-                      timeout_ns, wait_bias);
+        if (bytes * (size_t)nranks >= ((size_t)64 << 20))           // bandwidth-bound: trade registers for resident blocks
+            return launch(k_twoshot_flags<N, DT, 6>, grid, stream, pdl ? kLaunchPdl : kLaunchPlain, p, scratch, tile_flags, count,
+                          tv, lead_max, bw, timeout_ns, debug_bits);
+        return launch(k_twoshot_flags<N, DT, 4>, grid, stream, pdl ? kLaunchPdl : kLaunchPlain, p, scratch, tile_flags, count, tv,
+                      lead_max, bw, timeout_ns, debug_bits);
     });
 }
 
@@ -636,7 +640,8 @@ int launch_twoshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
         tile_flags = c->flags;
     }
     return launch_twoshot_flags(c->num_sms, o.blocks, p, nranks, dtype, count, (unsigned)std::max(0, o.twoshot_vecs), kMinFlagTileVec,
-                                scratch, tile_flags, c->bw, o.timeout_ns, (flags & NUNA_LAUNCH_PDL) != 0, 0u, stream);
+                                scratch, tile_flags, c->bw, o.timeout_ns, (flags & NUNA_LAUNCH_PDL) != 0,
+                                (o.keep_shard ? 4u : 0u) | ((flags & NUNA_TWOSHOT_SYS_SCOPE) ? 8u : 0u), stream);
 }
 
 int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, int dtype, size_t shard, unsigned flags,
@@ -704,8 +709,12 @@ int launch_alltoall(Context* c, const RankPtrs& p, int nranks, size_t block_byte
 
 // ---- single-kernel chain ---------------------------------------------------------------------------------
 
-// One cluster runs the whole chain, so it pays only while a node's work is small next to a kernel launch.
-constexpr size_t kChainPersistentMaxBytes = (size_t)128 << 10;     // per rank
+// One cluster runs the whole chain.  Measured on B200 (160 nodes, 8 ranks): 1.27 us per node at 16 KiB per rank
+// against 1.15 us for the graph with dependent launch, 5.8 against 1.4 us at 128 KiB: a node still costs two
+// dependent memory round trips (loads, then the stores the cluster barrier has to see performed) on sixteen
+// SMs, which is no less than a launch hidden behind its predecessor.  So the library never picks it by itself
+// (limit 0); NUNA_CHAIN_PERSISTENT runs it on request.
+constexpr size_t kChainPersistentMaxBytes = 0;                      // per rank
 
 bool chain_persistent_supported(const Context* c, int nsets, int nranks, int dtype, size_t count)
 {
@@ -831,7 +840,7 @@ int nuna_allreduce(const void* const* src, void* const* dst, int nranks, size_t 
                        : nranks <= 8 ? ((size_t)128 << 10) : ((size_t)64 << 10);
     constexpr size_t kSyncFactor = 8;
     const bool sync_form = (flags & NUNA_TWOSHOT_SYNC) && !(flags & NUNA_TWOSHOT_PUT);
-    const unsigned base = flags & ~(NUNA_TWOSHOT_SYNC | NUNA_TWOSHOT_PUT);
+    const unsigned base = flags & ~(NUNA_TWOSHOT_SYNC | NUNA_TWOSHOT_PUT | (sync_form ? 0u : NUNA_TWOSHOT_SYS_SCOPE));
     if (nranks <= 1 || bytes <= (sync_form ? limit * kSyncFactor : limit))
         return nuna_allreduce_oneshot(src, dst, nranks, count, dtype, base, stream);
     return nuna_allreduce_twoshot(src, dst, nranks, count, dtype, sync_form ? base : (base | NUNA_TWOSHOT_PUT), stream);
@@ -1054,14 +1063,65 @@ int nuna_debug_barrier_selftest(unsigned grid, unsigned expected, unsigned timeo
     return st;
 }
 
-/* Test hook: a flag-synchronised two-shot whose consumer items wait for a flag value that nobody publishes
- * (wait_bias = 1).  Every consumer wait runs out after timeout_ms, the kernel returns, destinations stay
- * unwritten and the status word latches NUNA_ERR_TIMEOUT -- nothing traps or hangs.                       */
-int nuna_debug_twoshot_unset_flags(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
-                                   unsigned timeout_ms)
+/* Measurement hook: one launch of the one-shot allreduce (8 ranks, bf16, whole vectors) under a placement --
+ * 0 round-robin, 1 co-located groups, 2 per-SM work lists -- with the latency of every work item's first load
+ * sampled per warp into hist[NUNA_DEBUG_LAT_BINS] (bins of NUNA_DEBUG_LAT_STEP cycles, added to what hist
+ * already holds).  Destinations receive the ordinary result.  Synchronises the device.                   */
+int nuna_debug_access_latency(const void* const* src, void* const* dst, size_t count, int placement, unsigned* hist)
+{
+    constexpr int N = 8;
+    int st = check_args(src, dst, N, count, count, NUNA_BF16, 0u, true);
+    if (st != NUNA_OK) return st;
+    if (!hist || count == 0 || count % 8 != 0 || placement < 0 || placement > 2) return NUNA_ERR_INVALID_ARG;
+    Context* c = nullptr;
+    if ((st = get_context(&c)) != NUNA_OK) return st;
+    const Options o = snapshot(c);
+    const RankPtrs p = make_ptrs(src, dst, N);
+    const size_t nvec = count / 8;
+    unsigned* d_hist = nullptr;
+    if (cudaMalloc(&d_hist, kLatBins * sizeof(unsigned)) != cudaSuccess) return NUNA_ERR_CUDA;
+    cudaMemset(d_hist, 0, kLatBins * sizeof(unsigned));
+    if (placement == 0) {
+        auto k = k_latency_rr<N, kBf16>;
+        const size_t ntiles = ceil_div(nvec, (size_t)kThreads);
+        st = launch(k, pick_grid(c, o, ntiles * N, NUNA_OCC(k)), (cudaStream_t)0, kLaunchPlain, p, count, ntiles, d_hist);
+    } else if (placement == 1) {
+        auto k = k_latency_group<N, 8, kBf16>;
+        const size_t ntiles = ceil_div(nvec, (size_t)(kThreads / 8));
+        st = launch(k, pick_grid(c, o, ntiles, NUNA_OCC(k)), (cudaStream_t)0, kLaunchPlain, p, count, ntiles, d_hist);
+    } else {
+        auto k = k_oneshot_sm<N, 8, kBf16, true>;
+        SmPlan pl;
+        st = get_sm_plan(c, N, nvec, 8, o.domains, (cudaStream_t)0, &pl);
+        if (st == NUNA_OK) {
+            SmLists sl;
+            sl.off = pl.off; sl.tiles = pl.tiles; sl.cursor = pl.cursor; sl.present = pl.present; sl.ctl = pl.ctl;
+            sl.nonempty = pl.nonempty; sl.num_sms = c->num_sms;
+            const size_t cap = (size_t)c->num_sms * (size_t)NUNA_OCC(k);
+            const unsigned grid = (unsigned)std::min(cap, std::max<size_t>((size_t)c->num_sms, (size_t)pl.total));
+            st = launch(k, grid, (cudaStream_t)0, kLaunchPlain, p, count, sl,
+                        (unsigned)std::max<size_t>(1, grid / (size_t)c->num_sms), d_hist);
+        }
+    }
+    if (st == NUNA_OK && cudaDeviceSynchronize() != cudaSuccess) st = NUNA_ERR_CUDA;
+    unsigned h[kLatBins];
+    if (st == NUNA_OK && cudaMemcpy(h, d_hist, sizeof h, cudaMemcpyDeviceToHost) != cudaSuccess) st = NUNA_ERR_CUDA;
+    if (st == NUNA_OK)
+        for (int b = 0; b < kLatBins; ++b) hist[b] += h[b];
+    cudaFree(d_hist);
+    return st;
+}
+
+/* Test hook: a flag-synchronised two-shot whose consumers wait for a flag value that nobody publishes
+ * (debug_bits = 1): every consumer wait runs out after timeout_ms, the kernel returns, destinations stay
+ * unwritten and the status word latches NUNA_ERR_TIMEOUT; nothing traps or hangs.  debug_bits = 0 is the
+ * ordinary kernel with an explicit timeout.                                                            */
+int nuna_debug_twoshot(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
+                       unsigned timeout_ms, unsigned debug_bits)
 {
     int st = check_args(src, dst, nranks, count, count, dtype, 0u, true);
     if (st != NUNA_OK || count == 0) return st;
+    if ((debug_bits & ~5u) != 0u) return NUNA_ERR_INVALID_ARG;
     Context* c = nullptr;
     if ((st = get_context(&c)) != NUNA_OK) return st;
     uint4* scratch;
@@ -1073,7 +1133,8 @@ int nuna_debug_twoshot_unset_flags(const void* const* src, void* const* dst, int
         tile_flags = c->flags;
     }
     return launch_twoshot_flags(c->num_sms, 0, make_ptrs(src, dst, nranks), nranks, dtype, count, 0u, kMinFlagTileVec, scratch,
-                                tile_flags, c->bw, (unsigned long long)timeout_ms * 1000000ull, false, 1u, (cudaStream_t)0);
+                                tile_flags, c->bw, (unsigned long long)timeout_ms * 1000000ull, false, debug_bits,
+                                (cudaStream_t)0);
 }
 
 }  // extern "C"

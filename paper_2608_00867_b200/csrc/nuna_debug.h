@@ -24,10 +24,20 @@ int nuna_debug_plan_oneshot(const nuna_topology_t* topo, int num_sms, int nranks
  * waits at most timeout_ms; writes how many blocks passed.  expected > grid makes the waits run out.    */
 int nuna_debug_barrier_selftest(unsigned grid, unsigned expected, unsigned timeout_ms, unsigned* passed);
 
-/* A flag-synchronised two-shot allreduce whose consumers wait for a flag value nobody publishes: every
- * wait runs out after timeout_ms, the kernel returns and the status word latches NUNA_ERR_TIMEOUT.     */
-int nuna_debug_twoshot_unset_flags(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
-                                   unsigned timeout_ms);
+/* The flag-synchronised two-shot allreduce with an explicit timeout.  debug_bits = 1: consumers wait for a
+ * flag value nobody publishes, so every wait runs out after timeout_ms, the kernel returns and the status
+ * word latches NUNA_ERR_TIMEOUT.                                                                        */
+int nuna_debug_twoshot(const void* const* src, void* const* dst, int nranks, size_t count, int dtype,
+                       unsigned timeout_ms, unsigned debug_bits);
+
+/* One launch of the one-shot allreduce (8 ranks, bf16, count a multiple of 8) under a placement -- 0 round-
+ * robin, 1 co-located groups, 2 per-SM work lists -- with the latency of every work item's first load sampled
+ * per warp: hist[b] += samples with latency in [b * NUNA_DEBUG_LAT_STEP, +NUNA_DEBUG_LAT_STEP) SM cycles, the last
+ * bin taking everything above.  The analogue of the paper's per-access latency distributions under its two
+ * placements (Section 6.2).  Destinations receive the ordinary result.  Synchronises the device.          */
+#define NUNA_DEBUG_LAT_BINS 64
+#define NUNA_DEBUG_LAT_STEP 32
+int nuna_debug_access_latency(const void* const* src, void* const* dst, size_t count, int placement, unsigned* hist);
 
 /* The probe's host-side clustering / verdict on a caller-supplied (num_sms x nlines) latency matrix.   */
 int nuna_debug_analyse_topology(const float* lat, const float* lat_rep, int num_sms, int nlines, nuna_topology_t* out);

@@ -38,6 +38,7 @@ struct Options {
     int domains = 0;                     // NUNA_DOMAINS: SM domains the work-list planner deals groups to (0 = what the probe found)
     int stage_vecs = 0;                  // NUNA_STAGE_VECS: vectors per source per tile of the staged one-shot (0 = by size)
     int twoshot_vecs = 0;                // NUNA_TWOSHOT_VECS: vectors per tile of the flag-synchronised two-shot (0 = by size)
+    int keep_shard = 0;                  // NUNA_KEEP_SHARD: do not discard consumed shard lines from L2 (measurement aid)
 };
 
 struct Context {
@@ -81,7 +82,7 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
 int launch_twoshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t count, unsigned flags, cudaStream_t stream);
 int launch_twoshot_flags(int num_sms, int blocks_override, const RankPtrs& p, int nranks, int dtype, size_t count,
                          unsigned tv, unsigned min_tv, uint4* scratch, unsigned* tile_flags, BarrierWords* bw,
-                         unsigned long long timeout_ns, bool pdl, unsigned wait_bias, cudaStream_t stream);
+                         unsigned long long timeout_ns, bool pdl, unsigned debug_bits, cudaStream_t stream);
 bool chain_persistent_pays_off(int dtype, size_t count);
 int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, int dtype, size_t shard, unsigned flags,
                           cudaStream_t stream);

@@ -222,17 +222,46 @@ __device__ __forceinline__ uint32_t load_elem_cg(const void* base, size_t elem)
     return w;
 }
 
+// ---- access-latency sampling (measurement builds of the one-shot kernels only) ----------------------------
+//
+// The timed variants below are the production loops with two clock reads around a work item's loads: t0
+// before the first load is issued, t1 once the first loaded vector can be used (a shared-memory store
+// consumes it, and instructions issue in order).  Lane 0 of every warp adds one sample per item to a
+// histogram of kLatBins bins of kLatStep cycles (the last bin also takes everything above): the
+// distribution of access latencies under a placement (Section 6.2).
+constexpr int kLatBins = 64, kLatStep = 32;
+
+__device__ __forceinline__ long long clock_now()
+{
+    long long t;
+    asm volatile("mov.u64 %0, %%clock64;" : "=l"(t) :: "memory");
+    return t;
+}
+
+__device__ __forceinline__ void latency_sample(unsigned* hist, long long t0, unsigned first_word)
+{
+    __shared__ unsigned sink[kThreads];
+    asm volatile("st.shared.u32 [%0], %1;" :: "r"((unsigned)__cvta_generic_to_shared(&sink[threadIdx.x])), "r"(first_word) : "memory");
+    const long long t1 = clock_now();
+    if ((threadIdx.x & 31u) == 0u) {
+        const long long bin = (t1 - t0) / kLatStep;
+        atomicAdd(hist + (bin < 0 ? 0 : bin >= kLatBins ? kLatBins - 1 : (int)bin), 1u);
+    }
+}
+
 // ---- one-shot allreduce: work item = (tile, destination rank) ---------------------------------
 //
 // Item i = tile * N + d, destination fastest, so the N emulated ranks that read
 // the same source tile are adjacent in the item order.  A tile is
 // kThreads * U vectors.  Round-robin placement: item i is taken by block
 // i mod gridDim.x (the locality-unaware baseline of Section 5.3).
-template <int N, int U, int DT>
-__device__ __forceinline__ void oneshot_item(const RankPtrs& p, size_t nvec, size_t tile, int d)
+template <int N, int U, int DT, bool kTimed = false>
+__device__ __forceinline__ void oneshot_item(const RankPtrs& p, size_t nvec, size_t tile, int d, unsigned* hist = nullptr)
 {
     const size_t base = tile * (size_t)(kThreads * U) + threadIdx.x;
     uint4 v[U][N];
+    long long t0 = 0;
+    if (kTimed) t0 = clock_now();
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const size_t i = base + (size_t)u * kThreads;
@@ -241,6 +270,7 @@ __device__ __forceinline__ void oneshot_item(const RankPtrs& p, size_t nvec, siz
             for (int r = 0; r < N; ++r) v[u][r] = ld_src(p.src[r] + i);
         }
     }
+    if (kTimed && base < nvec) latency_sample(hist, t0, v[0][0].x);
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const size_t i = base + (size_t)u * kThreads;
@@ -268,6 +298,17 @@ k_oneshot_rr(const RankPtrs p, const size_t count, const size_t ntiles)
     }
 }
 
+// The round-robin kernel's main loop with latency sampling (whole vectors only; a measurement aid).
+template <int N, int DT>
+__global__ void __launch_bounds__(kThreads, min_blocks(N))
+k_latency_rr(const RankPtrs p, const size_t count, const size_t ntiles, unsigned* hist)
+{
+    const size_t nvec = count / Elem<DT>::kElems;
+    const size_t nitems = ntiles * N;
+    for (size_t item = blockIdx.x; item < nitems; item += gridDim.x)
+        oneshot_item<N, 1, DT, true>(p, nvec, item / N, (int)(item % N), hist);
+}
+
 // ---- one-shot allreduce, co-located groups (placement-aware) ------------------------------------------
 //
 // Logical allocation (Section 4.2.1) puts the thread blocks that touch the same chunks into
@@ -291,18 +332,33 @@ __device__ __forceinline__ uint4 ld_src_l1(const uint4* p)
 // resource budget of Section 4.2.2 in SM terms: the more items of a group share an SM, the fewer
 // distinct bytes that SM has in flight (kThreads / C vectors per source), so cold data wants a small
 // C (more outstanding requests per SM) and L2-resident data a large one (fewer L2 -> SM transfers).
-template <int N, int C, int DT>
-__device__ __forceinline__ void oneshot_group(const RankPtrs& p, size_t nvec, size_t tile, int dst0)
+template <int N, int C, int DT, bool kTimed = false>
+__device__ __forceinline__ void oneshot_group(const RankPtrs& p, size_t nvec, size_t tile, int dst0, unsigned* hist = nullptr)
 {
     constexpr int kLanes = kThreads / C;                 // vectors per tile
     const int d = dst0 + threadIdx.x / kLanes;
     const size_t i = tile * kLanes + (threadIdx.x % kLanes);
     if (d < N && i < nvec) {
         uint4 v[N];
+        long long t0 = 0;
+        if (kTimed) t0 = clock_now();
 #pragma unroll
         for (int r = 0; r < N; ++r) v[r] = ld_src_l1(p.src[r] + i);
+        if (kTimed) latency_sample(hist, t0, v[0].x);
         st_dst(p.dst[d] + i, fold_vectors<N, DT>(v));
     }
+}
+
+// The co-located group kernel's main loop with latency sampling (whole vectors only; a measurement aid).
+template <int N, int C, int DT>
+__global__ void __launch_bounds__(kThreads, min_blocks(N))
+k_latency_group(const RankPtrs p, const size_t count, const size_t ntiles, unsigned* hist)
+{
+    constexpr int kSplit = (N + C - 1) / C;
+    const size_t nvec = count / Elem<DT>::kElems;
+    const size_t nitems = ntiles * kSplit;
+    for (size_t it = blockIdx.x; it < nitems; it += gridDim.x)
+        oneshot_group<N, C, DT, true>(p, nvec, it / kSplit, (int)(it % kSplit) * C, hist);
 }
 
 template <int N, int C, int DT>
@@ -582,9 +638,9 @@ __device__ __forceinline__ unsigned find_orphan(const SmLists& sl, unsigned own)
     return 0xFFFFFFFFu;
 }
 
-template <int N, int C, int DT>
+template <int N, int C, int DT, bool kTimed = false>
 __global__ void __launch_bounds__(kThreads, min_blocks(N))
-k_oneshot_sm(const RankPtrs p, const size_t count, const SmLists sl, const unsigned blocks_per_sm)
+k_oneshot_sm(const RankPtrs p, const size_t count, const SmLists sl, const unsigned blocks_per_sm, unsigned* hist)
 {
     pdl_wait();
     constexpr int kSplit = (N + C - 1) / C;
@@ -629,7 +685,7 @@ k_oneshot_sm(const RankPtrs p, const size_t count, const SmLists sl, const unsig
             for (unsigned i = 0; i < n; ++i) {
                 const size_t tile = sh_tiles[i];
 #pragma unroll
-                for (int sub = 0; sub < kSplit; ++sub) oneshot_group<N, C, DT>(p, nvec, tile, sub * C);
+                for (int sub = 0; sub < kSplit; ++sub) oneshot_group<N, C, DT, kTimed>(p, nvec, tile, sub * C, hist);
             }
         }
         __syncthreads();
@@ -890,19 +946,30 @@ __device__ __forceinline__ bool flag_barrier(BarrierWords* bw, unsigned int expe
 // every ticket of this launch is taken and stores (epoch + 1, 0) for the next launch.  Flags are compared
 // for equality with the epoch, so stale flags of earlier launches (or of another tiling) never match and
 // nothing is reset from the host.
-__device__ __forceinline__ void st_release(unsigned int* p, unsigned int v)
+// sys_scope: release / acquire at system scope, which is what the flags need once the ranks are separate
+// GPUs writing into each other's memory; within one GPU device scope is enough and cheaper.
+__device__ __forceinline__ void st_release(unsigned int* p, unsigned int v, bool sys_scope)
 {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+    if (sys_scope) asm volatile("st.release.sys.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+    else           asm volatile("st.release.gpu.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ unsigned int ld_acquire_scoped(const unsigned int* p, bool sys_scope)
+{
+    unsigned int v;
+    if (sys_scope) asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    else           asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 
 // Polls *flag until it equals `want`.  Returns false (and latches the timeout) when timeout_ns runs out.
 __device__ __forceinline__ bool wait_flag(const unsigned int* flag, unsigned int want, unsigned long long timeout_ns,
-                                          unsigned int* status)
+                                          unsigned int* status, bool sys_scope)
 {
-    if (ld_acquire(flag) == want) return true;
+    if (ld_acquire_scoped(flag, sys_scope) == want) return true;
     const unsigned long long t0 = globaltimer_ns();
     unsigned int polls = 0;
-    while (ld_acquire(flag) != want) {
+    while (ld_acquire_scoped(flag, sys_scope) != want) {
         if ((++polls & 63u) == 0u && globaltimer_ns() - t0 > timeout_ns) {
             atomicMax(status, 6u);                     // NUNA_ERR_TIMEOUT
             return false;
@@ -914,14 +981,27 @@ __device__ __forceinline__ bool wait_flag(const unsigned int* flag, unsigned int
 // Barrier among the 128 threads of one half of the block (ids 1 and 2; 0 is __syncthreads).
 __device__ __forceinline__ void half_sync(int id) { asm volatile("bar.sync %0, 128;" :: "r"(id) : "memory"); }
 
+// (Working ahead on the guess "my ticket will be my block index" while the ticket is on its way was tried
+// and measured slower: the blocks of a wave start together, so their tickets come back in no particular
+// order and most guesses are wrong.)
+//
 // tv: vectors per tile; shared memory = N * tv * 16 bytes.  lead_max: upper bound of `lead`.
-// wait_bias: 0 in normal use; a test passes 1 so that consumers wait for a value nobody publishes.
-template <int N, int DT>
-__global__ void __launch_bounds__(kThreads)
+// mode bits: 0 in normal use; bit 0: consumers wait for a flag value nobody publishes (test of the bounded
+// wait); bit 2: keep consumed shard lines in L2 (for measuring what the discard saves); bit 3: flags are
+// released and acquired at system scope (NUNA_TWOSHOT_SYS_SCOPE).
+// kMinBlocks: resident blocks per SM the register allocation is held to.  4 (64 registers) gives the shortest
+// path per block, best while the message is small enough for latency to dominate (8 KiB per rank: 3.4 us
+// against 3.7 us).  6 holds it to 40 registers: more tiles in flight per SM, which is what counts once the
+// message is bandwidth-bound (measured at 8 ranks: 16 MiB per rank 48.7 -> 45.6 us).
+template <int N, int DT, int kMinBlocks>
+__global__ void __launch_bounds__(kThreads, kMinBlocks)
 k_twoshot_flags(const RankPtrs p, uint4* scratch, unsigned int* flags, const size_t count, const unsigned tv,
-                const unsigned lead_max, BarrierWords* bw, const unsigned long long timeout_ns, const unsigned int wait_bias)
+                const unsigned lead_max, BarrierWords* bw, const unsigned long long timeout_ns, const unsigned int debug)
 {
     constexpr unsigned kHalf = kThreads / 2;
+    const unsigned wait_bias = debug & 1u;
+    const bool discard_shard = (debug & 4u) == 0u;
+    const bool sys_scope = (debug & 8u) != 0u;
     extern __shared__ __align__(128) unsigned char stage_raw[];
     uint4* stage = reinterpret_cast<uint4*>(stage_raw);            // [N][tv]
     __shared__ __align__(8) uint64_t bar;
@@ -974,13 +1054,14 @@ k_twoshot_flags(const RankPtrs p, uint4* scratch, unsigned int* flags, const siz
             half_sync(1);
             if (!landed) sh_landed = 0;
             half_sync(1);                              // every thread's shard stores are issued ...
-            if (threadIdx.x == 0 && sh_landed) st_release(flags + item, epoch1);   // ... and ordered before the flag
+            if (threadIdx.x == 0 && sh_landed) st_release(flags + item, epoch1, sys_scope);   // ... and ordered before the flag
         }
     } else {
         // ---- consume half ----
         if (consume) {
             const size_t ct = item - lead, cbase = ct * tv;
-            if (threadIdx.x == kHalf) sh_ok = wait_flag(flags + ct, epoch1 + wait_bias, timeout_ns, &bw->status) ? 1 : 0;
+            if (threadIdx.x == kHalf)
+                sh_ok = wait_flag(flags + ct, epoch1 + wait_bias, timeout_ns, &bw->status, sys_scope) ? 1 : 0;
             half_sync(2);                              // flag acquired by one thread -> every thread may read the tile
             if (sh_ok) {
                 const unsigned cnv = cbase < nvec ? (unsigned)((nvec - cbase < tv) ? nvec - cbase : tv) : 0u;
@@ -988,6 +1069,13 @@ k_twoshot_flags(const RankPtrs p, uint4* scratch, unsigned int* flags, const siz
                     const uint4 c = ld_cg(scratch + cbase + j);
 #pragma unroll
                     for (int d = 0; d < N; ++d) st_stream(p.dst[d] + cbase + j, c);
+                }
+                // The tile has exactly one consumer, so its shard lines are dead now: drop them from L2
+                // instead of letting them be written back to DRAM (whole, 128-byte aligned lines only).
+                if (discard_shard && (((uintptr_t)scratch | (uintptr_t)(cbase * 16u)) & 127u) == 0u) {
+                    half_sync(2);                      // every thread's loads of the tile have returned
+                    for (unsigned line = threadIdx.x - kHalf; line < cnv / 8u; line += kHalf)
+                        asm volatile("discard.global.L2 [%0], 128;" :: "l"(scratch + cbase + (size_t)line * 8u) : "memory");
                 }
                 if (ct == ntiles - 1 && tail0 < count) {
                     const size_t e = tail0 + (threadIdx.x - kHalf);

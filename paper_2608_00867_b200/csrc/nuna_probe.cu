@@ -26,6 +26,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <unordered_map>
 #include <vector>
 
 namespace nuna {
@@ -136,7 +137,8 @@ void sattolo_cycle(std::vector<unsigned>& next, uint64_t seed)
 
 // Splits SMs in two by the first principal component of the doubly-centred latency matrix and
 // fills the analysis fields of `out`.  lat[s * nlines + l], valid only for reported SMs.
-void analyse_topology(const std::vector<float>& lat, const std::vector<float>& lat_rep, int nlines, nuna_topology_t* out)
+void analyse_topology(const std::vector<float>& lat, const std::vector<float>& lat_rep, int nlines, nuna_topology_t* out,
+                      std::vector<int>* homes = nullptr)
 {
     std::vector<int> sms;
     for (int s = 0; s < out->num_sms && s < NUNA_MAX_SMS; ++s)
@@ -223,7 +225,8 @@ void analyse_topology(const std::vector<float>& lat, const std::vector<float>& l
     out->near_lat = (float)(near_sum / near_n);
     out->far_lat = (float)(far_sum / far_n);
     out->domain_gap = out->far_lat - out->near_lat;
-    for (int l = 0; l < L; ++l) out->line_home[l] = (unsigned char)home[l];
+    for (int l = 0; l < L && l < NUNA_MAX_PROBE_LINES; ++l) out->line_home[l] = (unsigned char)home[l];
+    if (homes) *homes = home;
     if (!(out->domain_gap > 3.0 * out->noise && out->domain_gap > 0.03 * median)) {
         for (int b = 0; b < NUNA_HIST_BINS; ++b) { out->hist_near[b] += out->hist_far[b]; out->hist_far[b] = 0; }
     } else {
@@ -314,9 +317,41 @@ int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
             }
         }
     }
+    const int nregular = (int)lines.size();
+    if (nregular < 2) return NUNA_ERR_INVALID_ARG;
+    out->num_lines = nregular;
+
+    // ---- address-granularity scan of buffer 0: a window of consecutive lines, and 16 sampled lines in each of
+    // up to eight consecutive blocks of 4 KiB, 64 KiB and 2 MiB.  A line is measured once; index_of maps an
+    // address to its row in the latency matrix.
+    std::unordered_map<uintptr_t, int> index_of;
+    for (int l = 0; l < nregular; ++l) index_of[(uintptr_t)lines[l]] = l;
+    auto line_index = [&](uintptr_t addr) {
+        auto it = index_of.find(addr);
+        if (it != index_of.end()) return it->second;
+        lines.push_back(reinterpret_cast<unsigned long long*>(addr));
+        index_of[addr] = (int)lines.size() - 1;
+        return (int)lines.size() - 1;
+    };
+    static const size_t kLevelBytes[NUNA_SCAN_LEVELS] = {(size_t)4 << 10, (size_t)64 << 10, (size_t)2 << 20};
+    std::vector<int> scan_idx;
+    std::vector<int> level_idx[NUNA_SCAN_LEVELS][NUNA_SCAN_BLOCKS];
+    {
+        const uintptr_t lo = ((uintptr_t)bufs[0] + 127) & ~(uintptr_t)127;
+        const uintptr_t hi = ((uintptr_t)bufs[0] + bytes[0]) & ~(uintptr_t)127;
+        const size_t nl = hi > lo ? (hi - lo) / 128 : 0;
+        const size_t window = std::min<size_t>(NUNA_SCAN_LINES, nl);
+        for (size_t i = 0; i < window; ++i) scan_idx.push_back(line_index(lo + i * 128));
+        for (int g = 0; g < NUNA_SCAN_LEVELS; ++g) {
+            const size_t per_block = kLevelBytes[g] / 128;
+            for (int b = 0; b < NUNA_SCAN_BLOCKS; ++b) {
+                if ((size_t)(b + 1) * per_block > nl) break;
+                for (int k = 0; k < 16; ++k)
+                    level_idx[g][b].push_back(line_index(lo + ((size_t)b * per_block + (size_t)(splitmix(seed) % per_block)) * 128));
+            }
+        }
+    }
     const int L = (int)lines.size();
-    if (L < 2) return NUNA_ERR_INVALID_ARG;
-    out->num_lines = L;
 
     // ---- device scratch ---------------------------------------------------------------------------------
     unsigned long long** d_lines = nullptr;
@@ -408,10 +443,45 @@ int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
         out->chain_walk_ok = walk_ok;
         out->chain_nodes = nnodes;
         out->chain_steps = kMissSteps;
-        analyse_topology(lat0, lat1, L, out);
+        std::vector<int> homes;
+        analyse_topology(lat0, lat1, L, out, &homes);
+        out->num_lines = nregular;
+        // granularity scan: runs of equal home among the consecutive lines, home shares per block size
+        for (int g = 0; g < NUNA_SCAN_LEVELS; ++g) {
+            out->scan_level_spread[g] = -1.f;
+            for (int b = 0; b < NUNA_SCAN_BLOCKS; ++b) out->scan_level_share[g][b] = -1.f;
+        }
+        if (out->verdict == NUNA_TOPO_NONUNIFORM && (int)homes.size() == L) {
+            out->scan_lines = (int)scan_idx.size();
+            int run = 0;
+            for (size_t i = 0; i < scan_idx.size(); ++i) {
+                out->scan_home[i] = (unsigned char)homes[scan_idx[i]];
+                ++run;
+                if (i + 1 == scan_idx.size() || homes[scan_idx[i + 1]] != homes[scan_idx[i]]) {
+                    out->scan_run_hist[std::min(run, NUNA_SCAN_RUN_BINS) - 1]++;
+                    out->scan_longest_run = std::max(out->scan_longest_run, run);
+                    run = 0;
+                }
+            }
+            for (int g = 0; g < NUNA_SCAN_LEVELS; ++g) {
+                float mn = 2.f, mx = -1.f;
+                int blocks = 0;
+                for (int b = 0; b < NUNA_SCAN_BLOCKS; ++b) {
+                    if (level_idx[g][b].empty()) continue;
+                    int h0 = 0;
+                    for (int li : level_idx[g][b]) h0 += homes[li] == 0;
+                    const float share = (float)h0 / (float)level_idx[g][b].size();
+                    out->scan_level_share[g][b] = share;
+                    mn = std::min(mn, share);
+                    mx = std::max(mx, share);
+                    ++blocks;
+                }
+                if (blocks >= 2) out->scan_level_spread[g] = mx - mn;
+            }
+        }
         // per (SM, buffer, region) mean hit latency and per (buffer, region) share of lines at home in domain 0
         std::vector<int> cnt((size_t)NUNA_MAX_PROBE_BUFS * NUNA_PROBE_REGIONS, 0), home0(cnt.size(), 0);
-        for (int l = 0; l < L; ++l) {
+        for (int l = 0; l < nregular; ++l) {
             const int idx = out->line_buf[l] * NUNA_PROBE_REGIONS + out->line_region[l];
             cnt[idx]++;
             home0[idx] += out->line_home[l] == 0;
@@ -425,7 +495,7 @@ int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
             if (!out->sm_reported[s]) continue;
             float sum[NUNA_MAX_PROBE_BUFS] = {};
             int n[NUNA_MAX_PROBE_BUFS] = {};
-            for (int l = 0; l < L; ++l) { sum[out->line_buf[l]] += lat0[(size_t)s * L + l]; n[out->line_buf[l]]++; }
+            for (int l = 0; l < nregular; ++l) { sum[out->line_buf[l]] += lat0[(size_t)s * L + l]; n[out->line_buf[l]]++; }
             for (int b = 0; b < nbufs; ++b) out->lat_hit[s][b] = n[b] ? sum[b] / n[b] : -1.f;
         }
         std::lock_guard<std::mutex> lock(c->mutex);

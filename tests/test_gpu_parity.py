@@ -59,7 +59,7 @@ COUNTS = [1, 7, 8, 9, 15, 16, 17, 2047, 2048, 2049, 4096, 6151, 100003, 262144]
 
 @pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16])
 @pytest.mark.parametrize("algo", ["oneshot", "oneshot_aware", "oneshot_staged", "oneshot_sm_lists", "twoshot", "twoshot_pdl",
-                                  "twoshot_put"])
+                                  "twoshot_sys", "twoshot_put"])
 def test_allreduce_special_values_all_counts(n, algo):
     for count in COUNTS:
         src = workloads.special_values(n, count, seed=1000 * n + count % 997)
@@ -74,7 +74,8 @@ def test_allreduce_special_values_all_counts(n, algo):
         elif algo == "oneshot_sm_lists":
             nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS)
         else:
-            f = {"twoshot": 0, "twoshot_pdl": nb.NUNA_LAUNCH_PDL, "twoshot_put": nb.NUNA_TWOSHOT_PUT}[algo]
+            f = {"twoshot": 0, "twoshot_pdl": nb.NUNA_LAUNCH_PDL, "twoshot_put": nb.NUNA_TWOSHOT_PUT,
+                 "twoshot_sys": nb.NUNA_TWOSHOT_SYS_SCOPE | nb.NUNA_LAUNCH_PDL}[algo]
             nb.nuna_allreduce_twoshot(dsrc, dst.view, count, flags=f)
         got = dst.numpy()
         for d in range(n):
@@ -607,7 +608,7 @@ def test_twoshot_ready_flag_wait_times_out_cleanly():
     nb.nuna_allreduce_twoshot(dsrc, dst.view, w.count)             # context, scratch and flags exist
     assert nb.nuna_device_status() == nb.NUNA_OK
     t0 = time.time()
-    assert nb.debug_twoshot_unset_flags(dsrc, dst.view, w.count, timeout_ms=50) == nb.NUNA_OK
+    assert nb.debug_twoshot(dsrc, dst.view, w.count, timeout_ms=50, unset_flags=True) == nb.NUNA_OK
     torch.cuda.synchronize()
     assert time.time() - t0 < 5.0                                  # bounded: nothing hangs
     assert nb.nuna_device_status() == nb.NUNA_ERR_TIMEOUT
@@ -617,6 +618,24 @@ def test_twoshot_ready_flag_wait_times_out_cleanly():
         nb.nuna_allreduce_twoshot(dsrc, dst.view, w.count, flags=flags)
         for got in dst.numpy():
             assert_same_bits(got, want, "two-shot after a timed-out launch")
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
+def test_access_latency_sampling_counts_every_item_and_keeps_the_result():
+    """The timed variants of the one-shot loops: one latency sample per warp and work item, every sample in a
+    plausible range, and the destinations still hold the oracle's bits."""
+    n, count = 8, 32 * 8192
+    src = workloads.special_values(n, count, seed=606)
+    want = oracle.allreduce(src, nthreads=4)[0]
+    dsrc = upload(src)
+    nvec = count // 8
+    for placement, warp_items in ((0, n * nvec // 32), (1, n * nvec // 32), (2, n * nvec // 32)):
+        dst = Dst(n, count)
+        hist = nb.debug_access_latency(dsrc, dst.view, count, placement, launches=2)
+        assert hist.sum() == 2 * warp_items, (placement, int(hist.sum()))
+        assert hist[0] == 0                                        # nothing returns in under 32 cycles
+        for got in dst.numpy():
+            assert_same_bits(got, want, f"timed placement {placement}")
     assert nb.nuna_device_status() == nb.NUNA_OK
 
 

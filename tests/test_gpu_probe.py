@@ -65,6 +65,35 @@ def test_verdict_is_consistent_with_its_own_numbers(probed):
         assert t.num_domains == 1 and not any(t.sm_domain[:t.num_sms])
 
 
+def test_granularity_scan_is_self_consistent_and_repeatable(probed):
+    """The consecutive-line scan of buffer 0: runs add up to the window, the histogram and the longest run
+    agree with the per-line homes, the block shares are shares, and a second probe maps the lines the same way."""
+    _, _, t1, t2 = probed
+    if t1.verdict != nb.NUNA_TOPO_NONUNIFORM:
+        assert t1.scan_lines == 0 and all(s == -1.0 for s in t1.scan_level_spread)
+        return
+    W = t1.scan_lines
+    assert W == min(nb.NUNA_SCAN_LINES, (1 << 19) // 128)       # buffer 0 is 512 KiB
+    homes = np.array(t1.scan_home[:W])
+    assert set(np.unique(homes)) <= {0, 1}
+    # run lengths recomputed from the homes
+    edges = np.flatnonzero(np.diff(homes)) + 1
+    runs = np.diff(np.concatenate([[0], edges, [W]]))
+    assert runs.sum() == W and runs.max() == t1.scan_longest_run
+    hist = np.bincount(np.minimum(runs, nb.NUNA_SCAN_RUN_BINS) - 1, minlength=nb.NUNA_SCAN_RUN_BINS)
+    assert np.array_equal(hist, np.array(t1.scan_run_hist[:]))
+    # block shares: 4 KiB and 64 KiB blocks fit in a 512 KiB buffer, 2 MiB blocks do not
+    for g, expect_blocks in ((0, 8), (1, 8), (2, 0)):
+        shares = [t1.scan_level_share[g][b] for b in range(nb.NUNA_SCAN_BLOCKS)]
+        got = [s for s in shares if s >= 0.0]
+        assert len(got) == expect_blocks and all(0.0 <= s <= 1.0 for s in got)
+        assert (t1.scan_level_spread[g] >= 0.0) == (expect_blocks >= 2)
+    # repeatable: the second probe puts (nearly) every line of the window in the same domain
+    assert t2.scan_lines == W
+    agree = (homes == np.array(t2.scan_home[:W])).mean()
+    assert agree >= 0.95, agree
+
+
 def test_probe_refuses_a_capturing_stream():
     buf = torch.zeros(4096, dtype=torch.int16, device="cuda")
     s = torch.cuda.Stream()
