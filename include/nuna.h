@@ -253,9 +253,14 @@ int nuna_init(size_t scratch_bytes);
  *                           more = every probed domain cut into equal latency quantiles; 0 = what the probe found
  *  NUNA_OPT_STAGE_VECS      16-byte vectors per source per tile of the NUNA_PLACE_STAGED kernel (0 = by size)
  *  NUNA_OPT_TWOSHOT_VECS    16-byte vectors per tile (= per ready flag) of the flag-synchronised two-shot (0 = by size)
+ *  NUNA_OPT_AG_BULK_VECS    nuna_allgather / nuna_alltoall move their (rank, tile) work items through the bulk-copy
+ *                           engine (one bulk load into shared memory, one bulk store per destination) by default (0,
+ *                           tile size by message size); >= 8: tiles of that many 16-byte vectors; 1: the register
+ *                           form instead (16-byte loads and stores by every thread)
  * Returns NUNA_ERR_INVALID_ARG for an unknown option or a negative value.  Creates the context.          */
 enum { NUNA_OPT_BLOCKS = 0, NUNA_OPT_UNROLL = 1, NUNA_OPT_COLOC = 2, NUNA_OPT_AUTO_MIN_BYTES = 3, NUNA_OPT_TIMEOUT_MS = 4,
-       NUNA_OPT_DOMAINS = 5, NUNA_OPT_STAGE_VECS = 6, NUNA_OPT_TWOSHOT_VECS = 7 };
+       NUNA_OPT_DOMAINS = 5, NUNA_OPT_STAGE_VECS = 6, NUNA_OPT_TWOSHOT_VECS = 7,
+       NUNA_OPT_AG_BULK_VECS = 8 };
 int nuna_set_option(int option, long long value);
 
 /* One-shot allreduce (Section 5.1, direct algorithm): every emulated rank d reads all N sources and

@@ -38,6 +38,7 @@ struct Options {
     int domains = 0;                     // NUNA_DOMAINS: SM domains the work-list planner deals groups to (0 = what the probe found)
     int stage_vecs = 0;                  // NUNA_STAGE_VECS: vectors per source per tile of the staged one-shot (0 = by size)
     int twoshot_vecs = 0;                // NUNA_TWOSHOT_VECS: vectors per tile of the flag-synchronised two-shot (0 = by size)
+    int ag_bulk_vecs = 0;                // NUNA_AG_BULK_VECS: > 0 = allgather through the bulk-copy engine with tiles of that many vectors
     int keep_shard = 0;                  // NUNA_KEEP_SHARD: do not discard consumed shard lines from L2 (measurement aid)
 };
 

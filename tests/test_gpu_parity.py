@@ -167,6 +167,31 @@ def test_reduce_scatter_and_allgather(n, shard, pdl):
         assert_same_bits(got_ag[d], got_ar[d], "ar vs ag(rs)")
 
 
+@pytest.mark.parametrize("bulk_vecs", [0, 1, 8, 2048])
+def test_allgather_and_alltoall_copy_forms(bulk_vecs):
+    """Bulk-copy form (default and extreme tile sizes) and register form of the two pure copies: raw bits,
+    ragged shard lengths, 16-byte-only alignment of the shards inside the destinations."""
+    rng = np.random.Generator(np.random.PCG64(17 + bulk_vecs))
+    try:
+        nb.nuna_set_option(nb.NUNA_OPT_AG_BULK_VECS, bulk_vecs)
+        for n, shard in ((16, 32768), (8, 8), (5, 2056), (3, 100000), (16, 24), (2, 300008)):
+            src = [rng.integers(0, 1 << 16, size=shard, dtype=np.uint32).astype(np.uint16) for _ in range(n)]
+            dst = Dst(n, n * shard)
+            nb.nuna_allgather(upload(src), dst.view, shard, flags=nb.NUNA_LAUNCH_PDL)
+            want = oracle.allgather(src)
+            for d, got in enumerate(dst.numpy()):
+                assert np.array_equal(got, want[d]), ("allgather", n, shard, d)
+            asrc = [rng.integers(0, 1 << 16, size=n * shard, dtype=np.uint32).astype(np.uint16) for _ in range(n)]
+            adst = Dst(n, n * shard)
+            nb.nuna_alltoall(upload(asrc), adst.view, shard)
+            awant = oracle.alltoall(asrc, nthreads=4)
+            for d, got in enumerate(adst.numpy()):
+                assert np.array_equal(got, awant[d]), ("alltoall", n, shard, d)
+    finally:
+        nb.nuna_set_option(nb.NUNA_OPT_AG_BULK_VECS, 0)
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
 def test_config_allgather16_raw_bits():
     w = workloads.config_allgather16()
     rng = np.random.Generator(np.random.PCG64(w.seed))
