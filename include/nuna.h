@@ -135,7 +135,7 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 #define NUNA_HIST_FIRST       200
 #define NUNA_HIST_STEP        4
 #define NUNA_SCAN_LINES       512   /* consecutive 128-byte lines of buffer 0 whose home domain is mapped      */
-#define NUNA_SCAN_RUN_BINS    16    /* run-length histogram: bin i = runs of i+1 lines, last bin = that or more */
+#define NUNA_SCAN_RUN_BINS    16    /* run-length histogram: bin b = runs of 2^b .. 2^(b+1)-1 lines               */
 #define NUNA_SCAN_LEVELS      3     /* granularities of the home-share table: 4 KiB, 64 KiB, 2 MiB             */
 #define NUNA_SCAN_BLOCKS      8     /* consecutive blocks of each granularity, from the start of buffer 0       */
 
@@ -173,7 +173,7 @@ typedef struct nuna_topology {
     /* At which granularity does the home domain of an address change (Section 3.2: latency depends on the
      * target address)?  scan_home[i] is the home domain of the i-th of scan_lines CONSECUTIVE 128-byte
      * lines of buffer 0 (from its first 128-byte boundary); scan_run_hist counts the runs of equal home
-     * among them by length, scan_longest_run is the longest.  scan_level_share[g][b] is the share of 16
+     * among them by length (power-of-two bins), scan_longest_run is the longest.  scan_level_share[g][b] is the share of 16
      * sampled lines at home in domain 0 inside the b-th consecutive block of 4 KiB (g = 0), 64 KiB (1) or
      * 2 MiB (2) of buffer 0, -1 where buffer 0 is too short; scan_level_spread[g] = max - min over the
      * blocks of that granularity (-1 with fewer than two blocks).  A spread near zero with shares near one

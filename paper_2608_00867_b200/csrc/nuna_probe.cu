@@ -458,7 +458,9 @@ int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
                 out->scan_home[i] = (unsigned char)homes[scan_idx[i]];
                 ++run;
                 if (i + 1 == scan_idx.size() || homes[scan_idx[i + 1]] != homes[scan_idx[i]]) {
-                    out->scan_run_hist[std::min(run, NUNA_SCAN_RUN_BINS) - 1]++;
+                    int bin = 0;
+                    while ((2 << bin) <= run && bin < NUNA_SCAN_RUN_BINS - 1) ++bin;     // 2^bin <= run < 2^(bin+1)
+                    out->scan_run_hist[bin]++;
                     out->scan_longest_run = std::max(out->scan_longest_run, run);
                     run = 0;
                 }

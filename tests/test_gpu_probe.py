@@ -80,7 +80,7 @@ def test_granularity_scan_is_self_consistent_and_repeatable(probed):
     edges = np.flatnonzero(np.diff(homes)) + 1
     runs = np.diff(np.concatenate([[0], edges, [W]]))
     assert runs.sum() == W and runs.max() == t1.scan_longest_run
-    hist = np.bincount(np.minimum(runs, nb.NUNA_SCAN_RUN_BINS) - 1, minlength=nb.NUNA_SCAN_RUN_BINS)
+    hist = np.bincount(np.floor(np.log2(runs)).astype(int), minlength=nb.NUNA_SCAN_RUN_BINS)     # power-of-two bins
     assert np.array_equal(hist, np.array(t1.scan_run_hist[:]))
     # block shares: 4 KiB and 64 KiB blocks fit in a 512 KiB buffer, 2 MiB blocks do not
     for g, expect_blocks in ((0, 8), (1, 8), (2, 0)):
