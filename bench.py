@@ -42,7 +42,8 @@ DTYPE = "bf16 storage, f32 accumulate"
 def PLACEMENT_VARIANTS(nb):
     """One-shot placements compared on the headline workload (flags of nuna_allreduce_oneshot)."""
     A = nb.NUNA_PLACE_AWARE
-    return {"roundrobin": nb.NUNA_PLACE_ROUNDROBIN, "aware_colocated": A, "aware_staged": A | nb.NUNA_PLACE_STAGED,
+    return {"roundrobin": nb.NUNA_PLACE_ROUNDROBIN, "aware_colocated_l1": A, "aware_staged_smem": A | nb.NUNA_PLACE_STAGED,
+            "aware_shared_regs": A | nb.NUNA_PLACE_REGS,
             "aware_cluster_dsmem": A | nb.NUNA_PLACE_CLUSTER, "aware_sm_lists": A | nb.NUNA_PLACE_SM_LISTS,
             "auto": nb.NUNA_PLACE_AUTO, "auto_resident_hint": nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT}
 
@@ -52,6 +53,7 @@ def CHAIN_VARIANTS(nb):
     P, G = nb.NUNA_LAUNCH_PDL, nb.NUNA_CHAIN_GRAPH
     return {"graph_roundrobin": G, "graph_roundrobin_pdl": G | P,
             "graph_aware_pdl": G | nb.NUNA_PLACE_AWARE | P,
+            "graph_regs_pdl": G | nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS | nb.NUNA_HINT_RESIDENT | P,
             "graph_staged_pdl": G | nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_STAGED | nb.NUNA_HINT_RESIDENT | P,
             "graph_auto_resident_pdl": G | nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT | P,
             "graph_sm_lists_pdl": G | nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS | P,
@@ -458,7 +460,7 @@ def run_gpu(args):
             return {"samples": tot, "mean_cycles": round(float((hist * mids).sum() / max(tot, 1)), 1), "p50_cycles": q(0.5),
                     "p95_cycles": q(0.95), "hist_step_cycles": nb.DEBUG_LAT_STEP, "hist": [int(x) for x in hist]}
         lat = {}
-        for pname, pl in (("roundrobin", 0), ("aware_colocated", 1), ("aware_sm_lists", 2)):
+        for pname, pl in (("roundrobin", 0), ("aware_colocated_l1", 1), ("aware_sm_lists", 2)):
             lat[pname] = {"l2_resident": lat_summary(nb.debug_access_latency(*sets[0], count, pl, launches=8)),
                           "cold": lat_summary(sum(nb.debug_access_latency(*sets[1 + i], count, pl) for i in range(len(sets) - 1)))}
         emit("first_load_latency_512KiB", lat)
@@ -531,6 +533,8 @@ def run_gpu(args):
         algos = {
             "oneshot": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, stream=st)),
             "oneshot_aware": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=nb.NUNA_PLACE_AWARE, stream=st)),
+            "oneshot_regs_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(
+                s, d, c, flags=P | nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS, stream=st)),
             "twoshot": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, stream=st)),
             "twoshot_put": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, flags=PUT, stream=st)),
             # the same with programmatic dependent launch
@@ -660,8 +664,9 @@ def run_gpu(args):
         summary["sweep"] = {
             "log2_bytes_per_rank": [r["bytes_per_rank"].bit_length() - 1 for r in sweep],
             "best_algo": [r["best"] for r in sweep],
-            "oneshot_us": [min(r["oneshot"]["cold_us"], r["oneshot_pdl"]["cold_us"], r["oneshot_auto_pdl"]["cold_us"],
-                               r["oneshot_staged_pdl"]["cold_us"]) for r in sweep],
+            "oneshot_roundrobin_us": [min(r["oneshot"]["cold_us"], r["oneshot_pdl"]["cold_us"]) for r in sweep],
+            "oneshot_auto_us": [r["oneshot_auto_pdl"]["cold_us"] for r in sweep],
+            "oneshot_staged_us": [r["oneshot_staged_pdl"]["cold_us"] for r in sweep],
             "twoshot_flag_us": flag_us,
             "twoshot_flag_frac": [round(2 * N_RANKS * r["bytes_per_rank"] / t / 1e3 / peak_gbs, 3) for r, t in zip(sweep, flag_us)],
             "twoshot_put_us": [min(r["twoshot_put"]["cold_us"], r["twoshot_put_pdl"]["cold_us"]) for r in sweep],
@@ -678,7 +683,7 @@ def run_gpu(args):
         "ms_per_step": round(us_per_step / 1e3, 7), "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": DTYPE, "data": "synthetic",
         "config": {"workload": w.name, "nranks": N_RANKS, "bytes_per_rank": w.bytes_per_rank,
-                   "algorithm": "one-shot, placement AUTO, PDL", "launch": f"graph of {m}x{K} calls per sample",
+                   "algorithm": "one-shot, placement AUTO (co-located group in registers), PDL", "launch": f"graph of {m}x{K} calls per sample",
                    "l2": f"cold, {len(sets)} buffer sets > 2xL2", "multi_gpu": "replicas only"},
         "replays": hs["samples"], "gpu_launches": int(launches_timed),
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak_gbs, "unit": "GB/s",

@@ -69,17 +69,17 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 #define NUNA_PLACE_AWARE      1u   /* a tile's N work items (one logical group, Section 4.2.1) are co-located:
                                       in one thread block by default, or through NUNA_PLACE_SM_LISTS /
                                       NUNA_PLACE_CLUSTER; only the one-shot allreduce distinguishes placements */
-#define NUNA_PLACE_AUTO       2u   /* the placement-aware kernel measured fastest for the size (co-located group
-                                      under NUNA_HINT_RESIDENT, shared-memory staged group for larger cold
-                                      messages), else exactly the ROUNDROBIN kernel                        */
+#define NUNA_PLACE_AUTO       2u   /* the placement-aware kernel measured fastest for the size (the co-located group
+                                      that shares its tile through registers, NUNA_PLACE_REGS, from 128 KiB per
+                                      rank), else exactly the ROUNDROBIN kernel                            */
 #define NUNA_PLACE_MASK       3u
 /* `flags`, bit 4 (nuna_allreduce_twoshot only): the reducing block stores its tile straight into all N
  * destinations, with no intermediate shard and no barrier.                                             */
 #define NUNA_TWOSHOT_PUT      16u
 /* `flags`, bit 5: hint that the sources were just written and are L2-resident (the decode case: a GEMM
- * epilogue produced them).  NUNA_PLACE_AUTO uses the placement-aware kernel only under this hint, from
- * 64 KiB per rank, and while 4 * nranks * bytes-per-rank fits in L2: the range where it was measured
- * to be at least as fast as the round-robin baseline.                                                  */
+ * epilogue produced them).  The register-sharing and shared-memory-staged one-shot kernels then co-locate
+ * all destinations of a tile (one fetch per tile) and store with the ordinary cache policy instead of
+ * evict-first.                                                                                          */
 #define NUNA_HINT_RESIDENT    32u
 /* `flags`, bit 6: launch with programmatic stream serialization.  The kernel may be scheduled while its
  * predecessor in the stream drains; it waits for that grid's completion and memory visibility before
@@ -121,6 +121,11 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
  * and the flags live in peer GPUs' memory (plain loads and stores through peer-mapped pointers).  Not tested
  * across GPUs.                                                                                          */
 #define NUNA_TWOSHOT_SYS_SCOPE 8192u
+/* `flags`, bit 14, with NUNA_PLACE_AWARE on nuna_allreduce_oneshot: the co-located group sharing the tile
+ * through registers.  The work items of C destinations (NUNA_OPT_COLOC: 2, 4 or 8) of one tile run in the
+ * same threads: a thread loads its vector of all N sources once and then does, for each of the C emulated
+ * ranks in turn, that rank's own rank-ordered fold and its store.                                        */
+#define NUNA_PLACE_REGS       16384u
 
 /* ---- topology probe --------------------------------------------------------------------------------
  * Result of nuna_probe_topology: caller-owned, plain data, fixed maximum sizes.  Latencies are in SM

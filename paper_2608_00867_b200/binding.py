@@ -35,6 +35,7 @@ NUNA_TWOSHOT_SYNC = 1024
 NUNA_CHAIN_PERSISTENT = 2048
 NUNA_CHAIN_GRAPH = 4096
 NUNA_TWOSHOT_SYS_SCOPE = 8192
+NUNA_PLACE_REGS = 16384
 
 NUNA_MAX_SMS, NUNA_MAX_PROBE_BUFS, NUNA_PROBE_REGIONS, NUNA_MAX_PROBE_LINES = 256, 32, 8, 2048
 NUNA_TOPO_UNIFORM, NUNA_TOPO_NONUNIFORM = 0, 1

@@ -116,7 +116,7 @@ int check_args(const void* const* src, void* const* dst, int nranks, size_t src_
     if (dtype != NUNA_BF16 && dtype != NUNA_F16 && dtype != NUNA_F32) return NUNA_ERR_UNSUPPORTED_DTYPE;
     if ((flags & ~(NUNA_PLACE_MASK | NUNA_TWOSHOT_PUT | NUNA_HINT_RESIDENT | NUNA_LAUNCH_PDL | NUNA_PLACE_SM_LISTS |
                    NUNA_PLACE_CLUSTER | NUNA_PLACE_STAGED | NUNA_TWOSHOT_SYNC | NUNA_CHAIN_PERSISTENT | NUNA_CHAIN_GRAPH |
-                   NUNA_TWOSHOT_SYS_SCOPE)) != 0u ||
+                   NUNA_TWOSHOT_SYS_SCOPE | NUNA_PLACE_REGS)) != 0u ||
         (flags & NUNA_PLACE_MASK) == 3u)
         return NUNA_ERR_INVALID_ARG;
     if (src_elems > ((size_t)1 << 40) || dst_elems > ((size_t)1 << 40)) return NUNA_ERR_TOO_LARGE;
@@ -291,21 +291,19 @@ static size_t ceil_div(size_t a, size_t b) { return (a + b - 1) / b; }
 // ---- collectives ---------------------------------------------------------------------------------
 
 // NUNA_PLACE_AUTO picks, per size, the one-shot kernel that was measured fastest on B200 (8 ranks; the
-// other rank counts use the same rules), never one that is slower than the round-robin baseline:
-//  * sources L2-resident (NUNA_HINT_RESIDENT) and 64 KiB <= bytes per rank, 4 N bytes within L2: the
-//    co-located group kernel (rows of one block share the tile through L1);
-//  * otherwise, from kStageMinBytes per rank: the group staged through shared memory by bulk copies;
-//  * otherwise the round-robin kernel itself.
-enum class OneShotKernel { RoundRobin, Group, Staged };
-constexpr size_t kStageMinBytes = (size_t)4 << 20;
+// other rank counts use the same rule), never one that is slower than the round-robin baseline: from
+// kRegsMinBytes per rank the co-located group that shares its tile through registers (cold, 8 ranks:
+// 256 KiB 2.14 vs 2.38 us, 512 KiB 2.76 vs 3.30, 4 MiB 11.5 vs 15.1, 64 MiB 157 vs 225; L2-resident 512 KiB
+// 1.72 vs 2.86), below that the round-robin kernel itself (8 KiB: 1.51 vs 1.58 us).  The other co-located
+// forms (through L1, through shared memory) are slower than this one at every size and stay opt-in.
+enum class OneShotKernel { RoundRobin, Group, Staged, Regs };
+constexpr size_t kRegsMinBytes = (size_t)128 << 10;
 
 static OneShotKernel auto_kernel(const Context* c, const Options& o, int nranks, size_t bytes, unsigned flags)
 {
+    (void)c; (void)flags;
     if (nranks < 2) return OneShotKernel::RoundRobin;
-    if ((flags & NUNA_HINT_RESIDENT) && 4 * bytes * (size_t)nranks <= c->l2_bytes && bytes >= o.auto_min_bytes)
-        return OneShotKernel::Group;
-    if (bytes >= kStageMinBytes) return OneShotKernel::Staged;
-    return OneShotKernel::RoundRobin;
+    return bytes >= std::max(kRegsMinBytes, o.auto_min_bytes) ? OneShotKernel::Regs : OneShotKernel::RoundRobin;
 }
 
 
@@ -505,6 +503,18 @@ static int launch_group(Context* c, const Options& o, const RankPtrs& p, size_t 
     return launch(k, grid, stream, mode, p, count, ntiles);
 }
 
+// Co-located group sharing the tile through registers: one (tile, C destinations) item per block.
+template <int N, int C, int DT>
+static int launch_regs(Context* c, const Options& o, const RankPtrs& p, size_t count, unsigned flags, unsigned mode, cudaStream_t stream)
+{
+    auto k = k_oneshot_regs<N, C, DT>;
+    const size_t nvec = count / Elem<DT>::kElems;
+    const size_t ntiles = ceil_div(nvec, (size_t)kThreads);
+    const size_t nitems = std::max<size_t>(ntiles * ((N + C - 1) / C), (count % Elem<DT>::kElems) ? (size_t)N : 0);
+    const unsigned grid = pick_grid(c, o, std::max<size_t>(nitems, 1), NUNA_OCC(k), 0);
+    return launch(k, grid, stream, mode, p, count, ntiles, (flags & NUNA_HINT_RESIDENT) ? 0 : 1);
+}
+
 // Staged group kernel: one tile per block.  Tile size (vectors per source): large enough that a tile's
 // N slices amortise the copy set-up, small enough that a mid-sized message still gives every SM several
 // blocks; 32 KiB of shared memory per block at most.
@@ -538,8 +548,25 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
     const size_t nvec = count / epv;
     const unsigned place = flags & NUNA_PLACE_MASK;
     OneShotKernel which = OneShotKernel::RoundRobin;
-    if (place == NUNA_PLACE_AWARE) which = (flags & NUNA_PLACE_STAGED) ? OneShotKernel::Staged : OneShotKernel::Group;
+    if (place == NUNA_PLACE_AWARE)
+        which = (flags & NUNA_PLACE_REGS) ? OneShotKernel::Regs : (flags & NUNA_PLACE_STAGED) ? OneShotKernel::Staged : OneShotKernel::Group;
     else if (place == NUNA_PLACE_AUTO) which = auto_kernel(c, o, nranks, bytes, flags);
+    if (which == OneShotKernel::Regs) {
+        const unsigned m = (flags & NUNA_LAUNCH_PDL) ? kLaunchPdl : kLaunchPlain;
+        // destinations per thread: four while the data comes from DRAM (two blocks per tile keep more loads in
+        // flight), all eight when it is L2-resident (one fetch per tile); measured at 8 ranks
+        int coloc = o.coloc > 0 ? o.coloc : ((flags & NUNA_HINT_RESIDENT) ? 8 : 4);
+        while (coloc > 2 && coloc / 2 >= nranks) coloc >>= 1;
+        // a small message needs its blocks more than it needs the sharing: keep at least half a wave of them
+        const size_t tiles = ceil_div(nvec, (size_t)kThreads);
+        while (o.coloc <= 0 && coloc > 2 && tiles * ceil_div((size_t)nranks, (size_t)coloc) < (size_t)c->num_sms / 2) coloc >>= 1;
+        return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
+            constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
+            if (coloc >= 8) return launch_regs<N, 8, DT>(c, o, p, count, flags, m, stream);
+            if (coloc >= 4) return launch_regs<N, 4, DT>(c, o, p, count, flags, m, stream);
+            return launch_regs<N, 2, DT>(c, o, p, count, flags, m, stream);
+        });
+    }
     if (which == OneShotKernel::Staged) {
         return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
             constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;

@@ -381,6 +381,107 @@ k_oneshot_group(const RankPtrs p, const size_t count, const size_t ntiles)
     }
 }
 
+// ---- one-shot allreduce, co-located group sharing the tile through registers -----------------------------
+//
+// The tightest co-location of a logical group: the work items (tile, d) of C destinations run in the SAME
+// threads.  A thread loads its vector of all N sources once and then performs, for each of the C emulated
+// ranks in turn, that rank's own fold in rank order and the store to that rank's destination.  The C folds
+// are separate instruction sequences (every addition is an opaque instruction, so the compiler cannot merge
+// the ranks' work into one); what the ranks share is the fetched data, as they share it through L1 in
+// k_oneshot_group and through shared memory in k_oneshot_stage -- here without a second trip through any
+// memory.  Loads and L2 -> SM traffic drop by C, the arithmetic stays N-fold.
+template <int DT>
+__device__ __forceinline__ float add_narrow_own(float acc, uint16_t h)
+{
+    float d;
+    if (DT == kBf16) asm volatile("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(acc));
+    else             asm volatile("add.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(acc));
+    return d;
+}
+
+__device__ __forceinline__ float add_f32_own(float a, float b)
+{
+    float d;
+    asm volatile("add.rn.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
+template <int DT>
+__device__ __forceinline__ void fold_word_own(float& lo, float& hi, uint32_t w)
+{
+    uint16_t l, h;
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(l), "=h"(h) : "r"(w));
+    lo = add_narrow_own<DT>(lo, l);
+    hi = add_narrow_own<DT>(hi, h);
+}
+
+// fold_vectors with additions the compiler must keep per call: same order, same instructions, same bits.
+template <int N, int DT>
+__device__ __forceinline__ uint4 fold_vectors_own(const uint4 (&v)[N])
+{
+    if (DT == kF32) {
+        float a0 = __uint_as_float(v[0].x), a1 = __uint_as_float(v[0].y);
+        float a2 = __uint_as_float(v[0].z), a3 = __uint_as_float(v[0].w);
+#pragma unroll
+        for (int r = 1; r < N; ++r) {
+            a0 = add_f32_own(a0, __uint_as_float(v[r].x));
+            a1 = add_f32_own(a1, __uint_as_float(v[r].y));
+            a2 = add_f32_own(a2, __uint_as_float(v[r].z));
+            a3 = add_f32_own(a3, __uint_as_float(v[r].w));
+        }
+        return make_uint4(__float_as_uint(a0), __float_as_uint(a1), __float_as_uint(a2), __float_as_uint(a3));
+    }
+    float a[8];
+    widen_word<DT>(a[0], a[1], v[0].x);
+    widen_word<DT>(a[2], a[3], v[0].y);
+    widen_word<DT>(a[4], a[5], v[0].z);
+    widen_word<DT>(a[6], a[7], v[0].w);
+#pragma unroll
+    for (int r = 1; r < N; ++r) {
+        fold_word_own<DT>(a[0], a[1], v[r].x);
+        fold_word_own<DT>(a[2], a[3], v[r].y);
+        fold_word_own<DT>(a[4], a[5], v[r].z);
+        fold_word_own<DT>(a[6], a[7], v[r].w);
+    }
+    return make_uint4(pack2<DT>(a[0], a[1]), pack2<DT>(a[2], a[3]), pack2<DT>(a[4], a[5]), pack2<DT>(a[6], a[7]));
+}
+
+// Work item = (tile of kThreads vectors, group of C destinations); one item per block.
+template <int N, int C, int DT>
+__global__ void __launch_bounds__(kThreads, min_blocks(N))
+k_oneshot_regs(const RankPtrs p, const size_t count, const size_t ntiles, const int stream_stores)
+{
+    pdl_wait();
+    constexpr int kSplit = (N + C - 1) / C;
+    const size_t nvec = count / Elem<DT>::kElems;
+    const size_t nitems = ntiles * kSplit;
+    for (size_t item = blockIdx.x; item < nitems; item += gridDim.x) {
+        const size_t i = (item / kSplit) * kThreads + threadIdx.x;
+        const int d0 = (int)(item % kSplit) * C;
+        if (i < nvec) {
+            uint4 v[N];
+#pragma unroll
+            for (int r = 0; r < N; ++r) v[r] = ld_src(p.src[r] + i);
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const int d = d0 + c;
+                if (d < N) {
+                    const uint4 o = fold_vectors_own<N, DT>(v);
+                    if (stream_stores) st_stream(p.dst[d] + i, o); else st_dst(p.dst[d] + i, o);
+                }
+            }
+        }
+    }
+    pdl_trigger();
+    const size_t tail0 = nvec * Elem<DT>::kElems;
+    if (tail0 < count) {
+        for (int d = blockIdx.x; d < N; d += gridDim.x) {
+            const size_t e = tail0 + threadIdx.x;
+            if (e < count) store_elem<DT>(p.dst[d], e, fold_scalar<N, DT>(p, e));
+        }
+    }
+}
+
 // ---- one-shot allreduce, co-located group staged through shared memory ---------------------------------
 //
 // The same logical group as above (one tile, every destination, on one compute unit), but the N

@@ -64,7 +64,7 @@ def test_validation_happens_before_any_cuda_call():
     assert call(ok_src, [A + 8192, A + 8192 + 16], 5, dtype=nb.NUNA_BF16) in (nb.NUNA_ERR_CUDA, nb.NUNA_OK)  # 10 bytes: fine
     assert call(ok_src, ok_dst, 8, dtype=77) == nb.NUNA_ERR_UNSUPPORTED_DTYPE
     assert call(ok_src, ok_dst, 8, flags=3) == nb.NUNA_ERR_INVALID_ARG
-    assert call(ok_src, ok_dst, 8, flags=1 << 14) == nb.NUNA_ERR_INVALID_ARG
+    assert call(ok_src, ok_dst, 8, flags=1 << 15) == nb.NUNA_ERR_INVALID_ARG
     assert call(ok_src, ok_dst, 8, flags=nb.NUNA_CHAIN_PERSISTENT) == nb.NUNA_ERR_INVALID_ARG    # chain-only bit
     assert call(ok_src, [A + 8192, 0], 8) == nb.NUNA_ERR_INVALID_ARG
     assert call(ok_src, [A + 8192, A + 12288 + 2], 8) == nb.NUNA_ERR_ALIGNMENT

@@ -46,9 +46,15 @@ ALGOS = {
     "oneshot_aware": lambda s, d, c, dt: nb.nuna_allreduce_oneshot(s, d, c, dtype=dt, flags=nb.NUNA_PLACE_AWARE),
     "oneshot_cluster": lambda s, d, c, dt: nb.nuna_allreduce_oneshot(s, d, c, dtype=dt,
                                                                     flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_CLUSTER),
+    "oneshot_staged": lambda s, d, c, dt: nb.nuna_allreduce_oneshot(s, d, c, dtype=dt,
+                                                                   flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_STAGED),
+    "oneshot_regs": lambda s, d, c, dt: nb.nuna_allreduce_oneshot(s, d, c, dtype=dt,
+                                                                 flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS | nb.NUNA_LAUNCH_PDL),
     "oneshot_sm_lists": lambda s, d, c, dt: nb.nuna_allreduce_oneshot(s, d, c, dtype=dt,
                                                                      flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS),
     "twoshot": lambda s, d, c, dt: nb.nuna_allreduce_twoshot(s, d, c, dtype=dt),
+    "twoshot_pdl_sys": lambda s, d, c, dt: nb.nuna_allreduce_twoshot(s, d, c, dtype=dt,
+                                                                    flags=nb.NUNA_LAUNCH_PDL | nb.NUNA_TWOSHOT_SYS_SCOPE),
     "twoshot_put": lambda s, d, c, dt: nb.nuna_allreduce_twoshot(s, d, c, dtype=dt, flags=nb.NUNA_TWOSHOT_PUT),
     "twoshot_static": lambda s, d, c, dt: nb.nuna_allreduce_twoshot_static(s, d, c, dtype=dt),
 }

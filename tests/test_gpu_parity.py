@@ -58,8 +58,8 @@ COUNTS = [1, 7, 8, 9, 15, 16, 17, 2047, 2048, 2049, 4096, 6151, 100003, 262144]
 
 
 @pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16])
-@pytest.mark.parametrize("algo", ["oneshot", "oneshot_aware", "oneshot_staged", "oneshot_sm_lists", "twoshot", "twoshot_pdl",
-                                  "twoshot_sys", "twoshot_put"])
+@pytest.mark.parametrize("algo", ["oneshot", "oneshot_aware", "oneshot_staged", "oneshot_regs", "oneshot_sm_lists", "twoshot",
+                                  "twoshot_pdl", "twoshot_sys", "twoshot_put"])
 def test_allreduce_special_values_all_counts(n, algo):
     for count in COUNTS:
         src = workloads.special_values(n, count, seed=1000 * n + count % 997)
@@ -71,6 +71,8 @@ def test_allreduce_special_values_all_counts(n, algo):
             nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE)
         elif algo == "oneshot_staged":
             nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_STAGED)
+        elif algo == "oneshot_regs":
+            nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS)
         elif algo == "oneshot_sm_lists":
             nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS)
         else:
@@ -127,7 +129,8 @@ def test_config_small_two_ranks():
 
 
 @pytest.mark.parametrize("flags", [nb.NUNA_PLACE_ROUNDROBIN, nb.NUNA_PLACE_AWARE, nb.NUNA_PLACE_AUTO,
-                                   nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT, nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_STAGED])
+                                   nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT, nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_STAGED,
+                                   nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS | nb.NUNA_LAUNCH_PDL])
 def test_config_decode_activation_all_placements(flags):
     w = workloads.config_decode_activation()
     src = workloads.make(w)
@@ -261,6 +264,7 @@ def test_full_size_64MiB_every_column_and_invariants():
     P = nb.NUNA_LAUNCH_PDL
     for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE),
                         (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_STAGED | P),
+                        (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS | P),
                         (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AUTO | P),
                         (nb.nuna_allreduce_twoshot, 0), (nb.nuna_allreduce_twoshot, P),
                         (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT | P), (nb.nuna_allreduce, 0)):
@@ -487,6 +491,7 @@ def test_tuning_options_change_the_launch_not_the_bits():
             for v in values:
                 nb.nuna_set_option(opt, v)
                 for call, flags in ((nb.nuna_allreduce_oneshot, 0), (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE),
+                                    (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS),
                                     (nb.nuna_allreduce_twoshot, 0), (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT)):
                     dst = Dst(w.nranks, w.count + 5)
                     call(dsrc, dst.view, w.count + 5, flags=flags)

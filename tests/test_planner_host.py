@@ -175,3 +175,37 @@ def test_lists_agree_with_the_python_oracle():
 def test_no_probe_means_one_domain_in_sm_order():
     lists = nb.debug_plan_oneshot(None, 10, 8, 25, 512, generic=True)
     assert lists == [[0, 1, 2], [3, 4, 5], [6, 7, 8], [9, 10, 11], [12, 13, 14], [15, 16, 17], [18, 19, 20], [21, 22, 23], [24], []]
+
+
+@pytest.mark.parametrize("domains", [1, 2, 4, 8, 16])
+@pytest.mark.parametrize("split", [True, False])
+def test_more_domains_than_probed_are_latency_quantiles(domains, split):
+    """NUNA_OPT_DOMAINS (the paper's sweep over the number of routing domains, Section 6.5): each probed
+    domain is cut into equal latency quantiles; group t goes to domain t mod D; closed form = general planner."""
+    num_sms, nranks, ntiles = 148, 8, 592
+    topo = fake_topology(num_sms, split, seed=11)
+    a = nb.debug_plan_oneshot(topo, num_sms, nranks, ntiles, 512, generic=True, domains=domains)
+    b = nb.debug_plan_oneshot(topo, num_sms, nranks, ntiles, 512, generic=False, domains=domains)
+    assert a == b
+    assert sorted(t for lst in a for t in lst) == list(range(ntiles))        # every tile exactly once
+    base = 2 if (split and domains != 1) else 1
+    D = max(base, domains // base * base) if domains > base else base
+    # an SM serves tiles of exactly one residue class mod D, and every class is served
+    classes = set()
+    for lst in a:
+        if lst:
+            assert len({t % D for t in lst}) == 1
+            classes.add(lst[0] % D)
+    assert classes == set(range(D))
+    # quantiles: inside a probed domain, the SMs of a faster class are never slower than those of a slower class
+    if D > base:
+        sub = D // base
+        for bdom in range(base):
+            by_class = {}
+            for s, lst in enumerate(a):
+                if lst and (topo.sm_domain[s] if base == 2 else 0) == bdom:
+                    by_class.setdefault(lst[0] % D, []).append(topo.sm_lat_hit[s])
+            keys = sorted(by_class)
+            assert len(keys) == sub
+            for lo, hi in zip(keys, keys[1:]):
+                assert max(by_class[lo]) <= min(by_class[hi])
