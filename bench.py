@@ -687,7 +687,7 @@ def run_gpu(args):
                    "l2": f"cold, {len(sets)} buffer sets > 2xL2", "multi_gpu": "replicas only"},
         "replays": hs["samples"], "gpu_launches": int(launches_timed),
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak_gbs, "unit": "GB/s",
-                     "frac": round(achieved / peak_gbs, 4), "traffic": recorded_traffic("oneshot_n8_512KiB"),
+                     "frac": round(achieved / peak_gbs, 4), "traffic": recorded_traffic("oneshot_regs_n8_512KiB"),
                      "peak_source": peak_src},
         "floor_us": floors["graph_node_pdl_us"],
         "e2e": {"value": round(e2e["value"], 2), "unit": "us", "h2d_bytes_per_step": e2e["h2d_bytes_per_step"],
@@ -734,6 +734,7 @@ def run_case(args):
         "oneshot": lambda s, d: nb.nuna_allreduce_oneshot(s, d, count),
         "oneshot_aware": lambda s, d: nb.nuna_allreduce_oneshot(s, d, count, flags=nb.NUNA_PLACE_AWARE),
         "oneshot_staged": lambda s, d: nb.nuna_allreduce_oneshot(s, d, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_STAGED),
+        "oneshot_regs": lambda s, d: nb.nuna_allreduce_oneshot(s, d, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS),
         "oneshot_sm": lambda s, d: nb.nuna_allreduce_oneshot(s, d, count, flags=nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS),
         "twoshot": lambda s, d: nb.nuna_allreduce_twoshot(s, d, count),
         "twoshot_put": lambda s, d: nb.nuna_allreduce_twoshot(s, d, count, flags=nb.NUNA_TWOSHOT_PUT),
@@ -758,7 +759,7 @@ def main():
     ap.add_argument("--sweep-max", type=int, default=26)
     ap.add_argument("--case", default=None,
                     help="ALGO:LOG2BYTES[:LAUNCHES] -- run a few eager launches of one algorithm at one size and "
-                         "exit (for ncu captures); ALGO in oneshot, oneshot_aware, oneshot_staged, oneshot_sm, twoshot, "
+                         "exit (for ncu captures); ALGO in oneshot, oneshot_aware, oneshot_staged, oneshot_regs, oneshot_sm, twoshot, "
                          "twoshot_put, allgather")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -890,8 +890,11 @@ int nuna_allreduce(const void* const* src, void* const* dst, int nranks, size_t 
     // size; the flag-synchronised form is used instead when the caller asks for it (NUNA_TWOSHOT_SYNC),
     // from the size where it beats the one-shot (measured per rank count, kSyncFactor x the put crossover).
     const size_t bytes = count * elem_size(dtype);
-    const size_t limit = nranks <= 2 ? ((size_t)1 << 20) : nranks <= 4 ? ((size_t)512 << 10)
-                       : nranks <= 8 ? ((size_t)128 << 10) : ((size_t)64 << 10);
+    size_t limit = nranks <= 2 ? ((size_t)1 << 20) : nranks <= 4 ? ((size_t)512 << 10)
+                 : nranks <= 8 ? ((size_t)128 << 10) : ((size_t)64 << 10);
+    // with NUNA_PLACE_AUTO the one-shot side is the register-sharing kernel, which stays ahead of the put form
+    // up to 1 MiB per rank (8 ranks: 256 KiB 2.13 vs 2.28 us, 512 KiB 2.76 vs 2.83, 1 MiB 3.94 vs 3.96)
+    if ((flags & NUNA_PLACE_MASK) == NUNA_PLACE_AUTO) limit = std::max(limit, (size_t)1 << 20);
     constexpr size_t kSyncFactor = 8;
     const bool sync_form = (flags & NUNA_TWOSHOT_SYNC) && !(flags & NUNA_TWOSHOT_PUT);
     const unsigned base = flags & ~(NUNA_TWOSHOT_SYNC | NUNA_TWOSHOT_PUT | (sync_form ? 0u : NUNA_TWOSHOT_SYS_SCOPE));
