@@ -70,8 +70,9 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
                                       in one thread block by default, or through NUNA_PLACE_SM_LISTS /
                                       NUNA_PLACE_CLUSTER; only the one-shot allreduce distinguishes placements */
 #define NUNA_PLACE_AUTO       2u   /* the placement-aware kernel measured fastest for the size (the co-located group
-                                      that shares its tile through registers, NUNA_PLACE_REGS, from 128 KiB per
-                                      rank), else exactly the ROUNDROBIN kernel                            */
+                                      that shares its tile through registers, NUNA_PLACE_REGS, from 1 MiB of
+                                      sources in total at 8 ranks or more, 2 MiB below), else exactly the
+                                      ROUNDROBIN kernel                                                    */
 #define NUNA_PLACE_MASK       3u
 /* `flags`, bit 4 (nuna_allreduce_twoshot only): the reducing block stores its tile straight into all N
  * destinations, with no intermediate shard and no barrier.                                             */
@@ -250,8 +251,10 @@ int nuna_init(size_t scratch_bytes);
  *  NUNA_OPT_BLOCKS          cap on the grid size of every kernel (the paper's "number of thread blocks",
  *                           Section 6.5: few blocks vs many)
  *  NUNA_OPT_UNROLL          vectors per thread per work item (1, 2, 4; limited so that N * unroll <= 16)
- *  NUNA_OPT_COLOC           destinations of a tile that share a block in the placement-aware one-shot (2, 4, 8)
- *  NUNA_OPT_AUTO_MIN_BYTES  smallest message per rank for which NUNA_PLACE_AUTO may pick the aware kernel
+ *  NUNA_OPT_COLOC           destinations of a tile that share a block (co-located group, work lists) or a thread
+ *                           (NUNA_PLACE_REGS) in the placement-aware one-shot (2, 4, 8; 0 = by rank count and hint)
+ *  NUNA_OPT_AUTO_MIN_BYTES  NUNA_PLACE_AUTO never picks a placement-aware kernel below this many bytes per rank
+ *                           (on top of its measured crossover)
  *  NUNA_OPT_TIMEOUT_MS      limit of every in-kernel wait (ready flags, barrier, bulk-copy completion)
  *  NUNA_OPT_DOMAINS         number of SM domains the NUNA_PLACE_SM_LISTS planner deals groups to (the paper's
  *                           sweep over routing domains, Section 6.5): 1 = one domain, 2 = the probed split,

@@ -62,7 +62,7 @@ int get_context(Context** out)
         c->opt.timeout_ns = (unsigned long long)env_int("NUNA_TIMEOUT_MS", 1000) * 1000000ull;
         c->opt.blocks = env_int("NUNA_BLOCKS", 0);
         c->opt.unroll = env_int("NUNA_UNROLL", 0);
-        c->opt.auto_min_bytes = (size_t)env_int("NUNA_AUTO_MIN_BYTES", 64 << 10);
+        c->opt.auto_min_bytes = (size_t)env_int("NUNA_AUTO_MIN_BYTES", 0);
         c->opt.coloc = env_int("NUNA_COLOC", 0);
         c->opt.domains = env_int("NUNA_DOMAINS", 0);
         c->opt.stage_vecs = env_int("NUNA_STAGE_VECS", 0);
@@ -290,20 +290,23 @@ static size_t ceil_div(size_t a, size_t b) { return (a + b - 1) / b; }
 
 // ---- collectives ---------------------------------------------------------------------------------
 
-// NUNA_PLACE_AUTO picks, per size, the one-shot kernel that was measured fastest on B200 (8 ranks; the
-// other rank counts use the same rule), never one that is slower than the round-robin baseline: from
-// kRegsMinBytes per rank the co-located group that shares its tile through registers (cold, 8 ranks:
-// 256 KiB 2.14 vs 2.38 us, 512 KiB 2.76 vs 3.30, 4 MiB 11.5 vs 15.1, 64 MiB 157 vs 225; L2-resident 512 KiB
-// 1.72 vs 2.86), below that the round-robin kernel itself (8 KiB: 1.51 vs 1.58 us).  The other co-located
-// forms (through L1, through shared memory) are slower than this one at every size and stay opt-in.
+// NUNA_PLACE_AUTO picks, per size, the one-shot kernel that was measured fastest on B200, never one that is
+// slower than the round-robin baseline: the co-located group that shares its tile through registers once the
+// message is large enough for the saved re-reads to matter (cold, 8 ranks: 256 KiB 2.14 vs 2.38 us, 512 KiB
+// 2.76 vs 3.30, 4 MiB 11.5 vs 15.1, 64 MiB 157 vs 225; L2-resident 512 KiB 1.72 vs 2.86; 16 ranks: 128 KiB
+// 2.33 vs 3.07, 4 MiB 21.5 vs 45.8), below that the round-robin kernel itself (8 ranks, 8 KiB: 1.51 vs 1.58 us).
+// The crossover was measured at 2, 3, 4, 8 and 16 ranks: 1 MiB of sources in total from 8 ranks up, 2 MiB below
+// (4 ranks: 256 KiB per rank 1.81 vs 1.79 us, 512 KiB 2.04 vs 2.11).  The other co-located forms (through L1,
+// through shared memory) are slower than this one at every size and stay opt-in.
 enum class OneShotKernel { RoundRobin, Group, Staged, Regs };
-constexpr size_t kRegsMinBytes = (size_t)128 << 10;
 
 static OneShotKernel auto_kernel(const Context* c, const Options& o, int nranks, size_t bytes, unsigned flags)
 {
     (void)c; (void)flags;
     if (nranks < 2) return OneShotKernel::RoundRobin;
-    return bytes >= std::max(kRegsMinBytes, o.auto_min_bytes) ? OneShotKernel::Regs : OneShotKernel::RoundRobin;
+    const size_t total = bytes * (size_t)nranks;
+    const size_t from = nranks >= 8 ? ((size_t)1 << 20) : ((size_t)2 << 20);
+    return (total >= from && bytes >= o.auto_min_bytes) ? OneShotKernel::Regs : OneShotKernel::RoundRobin;
 }
 
 
@@ -553,9 +556,11 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
     else if (place == NUNA_PLACE_AUTO) which = auto_kernel(c, o, nranks, bytes, flags);
     if (which == OneShotKernel::Regs) {
         const unsigned m = (flags & NUNA_LAUNCH_PDL) ? kLaunchPdl : kLaunchPlain;
-        // destinations per thread: four while the data comes from DRAM (two blocks per tile keep more loads in
-        // flight), all eight when it is L2-resident (one fetch per tile); measured at 8 ranks
-        int coloc = o.coloc > 0 ? o.coloc : ((flags & NUNA_HINT_RESIDENT) ? 8 : 4);
+        // destinations per thread: half of them while the data comes from DRAM (two blocks per tile keep more loads
+        // in flight), all of them (eight at most) when it is L2-resident (one fetch per tile)
+        // (measured at 2-16 ranks: 16 ranks x 4 MiB cold 21.5 us with eight destinations per thread, 24.0 with four)
+        const int all = std::min(8, pow2_at_least(nranks));
+        int coloc = o.coloc > 0 ? o.coloc : ((flags & NUNA_HINT_RESIDENT) ? all : std::min(8, std::max(2, pow2_at_least(nranks) / 2)));
         while (coloc > 2 && coloc / 2 >= nranks) coloc >>= 1;
         // a small message needs its blocks more than it needs the sharing: keep at least half a wave of them
         const size_t tiles = ceil_div(nvec, (size_t)kThreads);
@@ -837,7 +842,7 @@ int nuna_set_option(int option, long long value)
         case NUNA_OPT_BLOCKS: c->opt.blocks = (int)std::min<long long>(value, 1 << 22); break;
         case NUNA_OPT_UNROLL: c->opt.unroll = (int)value; break;
         case NUNA_OPT_COLOC: c->opt.coloc = (int)value; break;
-        case NUNA_OPT_AUTO_MIN_BYTES: c->opt.auto_min_bytes = value ? (size_t)value : ((size_t)64 << 10); break;
+        case NUNA_OPT_AUTO_MIN_BYTES: c->opt.auto_min_bytes = (size_t)value; break;
         case NUNA_OPT_TIMEOUT_MS: c->opt.timeout_ns = (unsigned long long)(value ? value : 1000) * 1000000ull; break;
         case NUNA_OPT_DOMAINS: c->opt.domains = (int)std::min<long long>(value, NUNA_MAX_SMS); break;
         case NUNA_OPT_STAGE_VECS: c->opt.stage_vecs = (int)std::min<long long>(value, 4096); break;
