@@ -479,7 +479,8 @@ def run_gpu(args):
         inter = {}
         for lname, load in loads.items():
             row = {}
-            for pname, pflags in (("roundrobin", nb.NUNA_PLACE_ROUNDROBIN), ("aware", nb.NUNA_PLACE_AWARE)):
+            for pname, pflags in (("roundrobin", nb.NUNA_PLACE_ROUNDROBIN), ("aware_l1", nb.NUNA_PLACE_AWARE),
+                                  ("auto_resident", nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT)):
                 fn = lambda s, d, st, f=pflags: nb.nuna_allreduce_oneshot(s, d, c1, flags=f, stream=st)
                 g = capture(fn, isets, 400)
                 with torch.cuda.stream(stream):
