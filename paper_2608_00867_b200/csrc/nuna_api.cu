@@ -624,11 +624,14 @@ int launch_twoshot_flags(int num_sms, int blocks_override, const RankPtrs& p, in
     const size_t bytes = count * elem_size(dtype);
     const size_t nvec = count / elems_per_vec(dtype);
     if (tv == 0) {
-        // tile bytes across all N sources: small tiles while the message is small (more blocks, less latency
-        // per tile), up to 32 KiB once there are plenty of tiles
+        // Tile bytes across all N sources, from a sweep at 8 ranks (16 ... 256 vectors per tile at every size):
+        // small tiles while the message is small (more blocks, less latency per tile), 32 KiB once there are
+        // plenty.  At 8 MiB of sources 16 KiB tiles make 1024 blocks for 592 resident ones and the second
+        // wave's consumers wait (10.3 us against 7.6 us with 12 KiB tiles), hence the step back there.
         const size_t src_bytes = bytes * (size_t)nranks;
-        const unsigned tile_src = src_bytes <= ((size_t)1 << 20) ? 4096u : src_bytes <= ((size_t)8 << 20) ? 8192u
-                                : src_bytes <= ((size_t)64 << 20) ? 16384u : 32768u;
+        const unsigned tile_src = src_bytes <= ((size_t)512 << 10) ? 4096u : src_bytes <= ((size_t)1 << 20) ? 8192u
+                                : src_bytes <= ((size_t)4 << 20) ? 16384u : src_bytes <= ((size_t)8 << 20) ? 12288u
+                                : src_bytes <= ((size_t)32 << 20) ? 16384u : 32768u;
         tv = tile_src / 16u / (unsigned)nranks;
     }
     tv = std::max(min_tv, std::min(tv, 2048u / (unsigned)nranks));

@@ -54,6 +54,22 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point():
     assert all(torch.equal(r, g) for r, g in zip(ref, got))
 
 
+def test_device_memory_in_use_does_not_change():
+    """The entry point exists for callers that must not allocate: after the first call on the device, further
+    calls of any size leave the amount of free device memory exactly where it was."""
+    n = 4
+    bufs = {c: ([torch.zeros(c, dtype=torch.int16, device="cuda") for _ in range(n)],
+                [torch.zeros(c, dtype=torch.int16, device="cuda") for _ in range(n)]) for c in (8, 4099, 1 << 20)}
+    nb.nuna_allreduce_twoshot_static(*bufs[8], 8)                # first call on the device: set-up, no allocation either
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for _ in range(3):
+        for c, (src, dst) in bufs.items():
+            nb.nuna_allreduce_twoshot_static(src, dst, c)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+
+
 def test_sizes_beyond_the_fixed_array_are_refused():
     n = 2
     count = nb.NUNA_STATIC_MAX_COUNT + 8
