@@ -15,8 +15,9 @@ Output: every detail section (message-size sweep 8 KiB ... 64 MiB per rank with 
 two-shot and put variants, cold and warm, isolated per-call latencies, launch floors, the
 16-rank allgather, reduce-scatter, alltoall, the 160-node decode chain, probe summary,
 placement, domain-count and block-count sensitivity, interference) is printed on its own
-stdout line as it completes and collected in gpurun_out/bench_detail.json; the LAST stdout
-line is the compact result object.
+stdout line as it completes and collected in bench_detail.json (in the directory named by
+BENCH_OUT_DIR, by default the run's output folder); the LAST stdout line is the compact result
+object.
 """
 from __future__ import annotations
 
@@ -704,7 +705,7 @@ def run_gpu(args):
     if cpu is not None:
         line["cpu_baseline"] = cpu
     try:
-        out_dir = os.path.join(ROOT, "gpurun_out")
+        out_dir = os.path.join(ROOT, os.environ.get("BENCH_OUT_DIR", "gpurun_out"))
         os.makedirs(out_dir, exist_ok=True)
         with open(os.path.join(out_dir, "bench_detail.json"), "w") as f:
             json.dump({"result": line, "detail": detail}, f, indent=1)

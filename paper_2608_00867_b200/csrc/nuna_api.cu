@@ -776,11 +776,11 @@ int launch_alltoall(Context* c, const RankPtrs& p, int nranks, size_t block_byte
 
 // ---- single-kernel chain ---------------------------------------------------------------------------------
 
-// One cluster runs the whole chain.  Measured on B200 (160 nodes, 8 ranks): 1.27 us per node at 16 KiB per rank
-// against 1.15 us for the graph with dependent launch, 5.8 against 1.4 us at 128 KiB: a node still costs two
-// dependent memory round trips (loads, then the stores the cluster barrier has to see performed) on sixteen
-// SMs, which is no less than a launch hidden behind its predecessor.  So the library never picks it by itself
-// (limit 0); NUNA_CHAIN_PERSISTENT runs it on request.
+// One cluster runs the whole chain.  Measured on B200 (160 nodes, 8 ranks): 1.45 us per node at 16 KiB per rank
+// against 1.13-1.15 us for the graph with dependent launch, 2.5 against 1.3 us at 128 KiB, 12 against 2.5 us at
+// 1 MiB: a node still costs two dependent memory round trips (loads; then the stores the cluster barrier has to
+// see performed) plus the barrier on sixteen SMs, which is no less than a launch hidden behind its predecessor.
+// So the library never picks it by itself (limit 0); NUNA_CHAIN_PERSISTENT runs it on request.
 constexpr size_t kChainPersistentMaxBytes = 0;                      // per rank
 
 bool chain_persistent_supported(const Context* c, int nsets, int nranks, int dtype, size_t count)
@@ -795,9 +795,12 @@ int launch_chain_persistent(Context* c, const ChainSets& sets, int nsets, int nn
                             cudaStream_t stream)
 {
     (void)c;
+    // two destinations per thread while that still gives every thread of the cluster an item, all of them beyond
+    const bool wide = (count / elems_per_vec(dtype)) * (size_t)((nranks + 1) / 2) > (size_t)16 * kThreads;
     return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
         constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
-        auto k = k_chain_persistent<N, DT>;
+        constexpr int kAll = pow2_at_least(N) > 8 ? 8 : (pow2_at_least(N) < 2 ? 2 : pow2_at_least(N));
+        auto k = wide ? k_chain_persistent<N, kAll, DT> : k_chain_persistent<N, 2, DT>;
         // sixteen blocks per cluster need the non-portable opt-in; fall back to the portable eight
         static std::atomic<int> cluster_size[kMaxDevices];
         int dev = 0;
@@ -805,7 +808,8 @@ int launch_chain_persistent(Context* c, const ChainSets& sets, int nsets, int nn
         int cs = cluster_size[dev].load(std::memory_order_relaxed);
         if (cs == 0) {
             cs = 8;
-            if (cudaFuncSetAttribute(k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+            if (cudaFuncSetAttribute(k_chain_persistent<N, kAll, DT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+                cudaFuncSetAttribute(k_chain_persistent<N, 2, DT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
                 cudaLaunchConfig_t cfg = {};
                 cfg.gridDim = dim3(16, 1, 1);
                 cfg.blockDim = dim3(kThreads, 1, 1);

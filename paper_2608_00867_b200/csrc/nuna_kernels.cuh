@@ -1308,9 +1308,9 @@ k_twoshot_put(const RankPtrs p, const size_t count, const size_t ntiles)
 // times the data time, so the whole chain of back-to-back one-shot allreduces runs as ONE kernel on one
 // thread-block cluster.  Node k works on buffer set k mod nsets; the node boundary is a cluster barrier
 // with release / acquire semantics, so node k+1 reads only after every block has finished writing node k
-// (a node may read what its predecessor wrote).  Within a node the work is the co-located one-shot:
-// block b takes tiles b, b + blocks, ...; row d of a block is emulated rank d's item for that tile.
-// Loads are ordinary coherent global loads (a source may have been written by the previous node).
+// (a node may read what its predecessor wrote).  Within a node the work is the register-sharing co-located
+// one-shot, items dealt to the cluster's threads in order.  Loads go to L2 (ld.global.cg): a source may have
+// been written by another SM in the previous node, and L1 is not coherent between SMs.
 __device__ __forceinline__ unsigned cluster_nctarank()
 {
     unsigned r;
@@ -1326,56 +1326,42 @@ __device__ __forceinline__ uint4 ld_coherent(const uint4* p)
     return v;
 }
 
-template <int N, int DT>
+template <int N, int C, int DT>
 __global__ void __launch_bounds__(kThreads, 1)
 k_chain_persistent(const __grid_constant__ ChainSets sets, const int nsets, const int nnodes, const size_t count)
 {
-    constexpr int C = pow2_at_least(N) > 8 ? 8 : pow2_at_least(N);
-    constexpr int kLanes = kThreads / C;
-    constexpr int kSplit = (N + C - 1) / C;
+    constexpr int kSplit = (N + C - 1) / C;                // destination groups per vector
     const unsigned nblk = cluster_nctarank(), blk = cluster_ctarank();
     const size_t nvec = count / Elem<DT>::kElems;
-    const size_t nitems = ((nvec + kLanes - 1) / kLanes) * kSplit;
+    const size_t nitems = nvec * kSplit;                   // item = (vector, group of C destinations), group fastest
     const size_t tail0 = nvec * Elem<DT>::kElems;
-    const int row = threadIdx.x / kLanes, lane = threadIdx.x % kLanes;
+    const size_t first = (size_t)blk * kThreads + threadIdx.x, stride = (size_t)nblk * kThreads;
     int set = 0;
     for (int node = 0; node < nnodes; ++node) {
         const RankPtrs& p = sets.s[set];
-        // two items per step so that 2N loads are in flight per thread
-        for (size_t it = blk; it < nitems; it += 2 * (size_t)nblk) {
-            uint4 v[2][N];
-            size_t vi[2];
-            int dd[2];
+        // within a node the work is the register-sharing one-shot: N loads once, C rank-ordered folds and stores
+        for (size_t item = first; item < nitems; item += stride) {
+            const size_t i = item / kSplit;
+            const int d0 = (int)(item % kSplit) * C;
+            uint4 v[N];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const size_t item = it + (size_t)h * nblk;
-                dd[h] = (int)(item % kSplit) * C + row;
-                vi[h] = (item / kSplit) * kLanes + lane;
-                if (item < nitems && dd[h] < N && vi[h] < nvec) {
+            for (int r = 0; r < N; ++r) v[r] = ld_cg(p.src[r] + i);
 #pragma unroll
-                    for (int r = 0; r < N; ++r) v[h][r] = ld_coherent(p.src[r] + vi[h]);
-                } else {
-                    dd[h] = -1;
-                }
-            }
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-                if (dd[h] >= 0) st_dst(p.dst[dd[h]] + vi[h], fold_vectors<N, DT>(v[h]));
+            for (int c = 0; c < C; ++c)
+                if (d0 + c < N) st_dst(p.dst[d0 + c] + i, fold_vectors_own<N, DT>(v));
         }
         if (tail0 < count && blk == 0) {
-            const size_t e = tail0 + lane;
-            for (int d = row; d < N && e < count; d += C) {
+            const size_t e = tail0 + (threadIdx.x % 32);
+            for (int d = threadIdx.x / 32; d < N && e < count; d += kThreads / 32) {
                 uint32_t w;
                 if (DT == kF32) {
-                    float acc = __uint_as_float(*reinterpret_cast<const volatile uint32_t*>(reinterpret_cast<const uint32_t*>(p.src[0]) + e));
-                    for (int r = 1; r < N; ++r)
-                        acc = __fadd_rn(acc, __uint_as_float(*reinterpret_cast<const volatile uint32_t*>(reinterpret_cast<const uint32_t*>(p.src[r]) + e)));
+                    float acc = __uint_as_float(load_elem_cg<DT>(p.src[0], e));
+                    for (int r = 1; r < N; ++r) acc = __fadd_rn(acc, __uint_as_float(load_elem_cg<DT>(p.src[r], e)));
                     w = __float_as_uint(acc);
                 } else {
                     float acc, unused;
-                    widen_word<DT>(acc, unused, (uint32_t)*reinterpret_cast<const volatile uint16_t*>(reinterpret_cast<const uint16_t*>(p.src[0]) + e));
-                    for (int r = 1; r < N; ++r)
-                        acc = add_narrow<DT>(acc, *reinterpret_cast<const volatile uint16_t*>(reinterpret_cast<const uint16_t*>(p.src[r]) + e));
+                    widen_word<DT>(acc, unused, load_elem_cg<DT>(p.src[0], e));
+                    for (int r = 1; r < N; ++r) acc = add_narrow<DT>(acc, (uint16_t)load_elem_cg<DT>(p.src[r], e));
                     w = pack2<DT>(acc, 0.0f) & 0xFFFFu;
                 }
                 store_elem<DT>(p.dst[d], e, w);
