@@ -579,6 +579,26 @@ def run_gpu(args):
             del ssets
             torch.cuda.empty_cache()
 
+        # ---- other rank counts: the automatic choices against the round-robin baseline and the put form ------
+        ranks_rows = []
+        for n in (2, 4, 16):
+            for log2b in (17, 19, 22):
+                c = (1 << log2b) // 2
+                nsets = make_sets(n, c, c, 2 * l2 + (64 << 20), "normal", 90 + n)
+                nodes_n = max(len(nsets), min(512, (256 << 20) // ((1 << log2b) * n // 8 + 1) + 1))
+                row = {"nranks": n, "bytes_per_rank": 1 << log2b}
+                for name, fn in (("oneshot_roundrobin_pdl", lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=P, stream=st)),
+                                 ("oneshot_auto_pdl", lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=P | nb.NUNA_PLACE_AUTO, stream=st)),
+                                 ("twoshot_pdl", lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, flags=P, stream=st)),
+                                 ("twoshot_put_pdl", lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, flags=P | PUT, stream=st)),
+                                 ("selected_auto_pdl", lambda s, d, st: nb.nuna_allreduce(s, d, c, flags=P | nb.NUNA_PLACE_AUTO, stream=st))):
+                    row[name] = round(per_call_us(fn, nsets, nodes_n), 3)
+                row["best_frac_of_peak"] = round(2 * n * (1 << log2b) / min(v for k, v in row.items() if k.endswith("_pdl")) / 1e3 / peak_gbs, 4)
+                ranks_rows.append(row)
+                del nsets
+                torch.cuda.empty_cache()
+        emit("other_rank_counts_cold_us", ranks_rows)
+
         # ---- allgather, 16 ranks x 64 KiB ---------------------------------------------------------------
         wa = workloads.config_allgather16()
         asets = make_sets(wa.nranks, wa.count, wa.nranks * wa.count, 2 * l2 + (64 << 20), "uniform", wa.seed)
