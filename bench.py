@@ -438,6 +438,9 @@ def run_gpu(args):
             "far_cycles": round(topo.far_lat, 1), "gap_cycles": round(topo.domain_gap, 1), "noise_cycles": round(topo.noise, 2),
             "sm_mean_hit_cycles_min_max": [round(min(topo.sm_lat_hit[:topo.num_sms]), 1), round(max(topo.sm_lat_hit[:topo.num_sms]), 1)],
             "sm_miss_cycles_min_max": [round(min(topo.sm_lat_miss[:topo.num_sms]), 1), round(max(topo.sm_lat_miss[:topo.num_sms]), 1)],
+            "sm_solo_read_gbs_min_median_max": [round(float(x), 1) for x in np.percentile(np.array(topo.sm_read_gbs[:topo.num_sms]), [0, 50, 100])],
+            "sm_solo_read_gbs_median_by_domain": [round(float(np.median([topo.sm_read_gbs[s] for s in range(topo.num_sms) if doms[s] == dd] or [0])), 1)
+                                                  for dd in (0, 1)],
             "hist_first_cycle": nb.NUNA_HIST_FIRST, "hist_step": nb.NUNA_HIST_STEP,
             "hist_near": list(topo.hist_near), "hist_far": list(topo.hist_far),
             "scan": {"consecutive_lines": topo.scan_lines, "longest_run": topo.scan_longest_run,

@@ -67,8 +67,10 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 /* `flags`, bits 0-1: thread-block placement (Section 4.2 / Section 5.3 baseline). */
 #define NUNA_PLACE_ROUNDROBIN 0u   /* locality-unaware: work item i -> thread block i mod grid          */
 #define NUNA_PLACE_AWARE      1u   /* a tile's N work items (one logical group, Section 4.2.1) are co-located:
-                                      in one thread block by default, or through NUNA_PLACE_SM_LISTS /
-                                      NUNA_PLACE_CLUSTER; only the one-shot allreduce distinguishes placements */
+                                      in one thread block, sharing the tile through L1, by default; through
+                                      registers, shared memory, per-SM work lists or a cluster with
+                                      NUNA_PLACE_REGS / _STAGED / _SM_LISTS / _CLUSTER; only the one-shot
+                                      allreduce distinguishes placements                                   */
 #define NUNA_PLACE_AUTO       2u   /* the placement-aware kernel measured fastest for the size (the co-located group
                                       that shares its tile through registers, NUNA_PLACE_REGS, from 1 MiB of
                                       sources in total at 8 ranks or more, 2 MiB below), else exactly the
@@ -191,12 +193,17 @@ typedef struct nuna_topology {
     unsigned scan_run_hist[NUNA_SCAN_RUN_BINS];
     float scan_level_share[NUNA_SCAN_LEVELS][NUNA_SCAN_BLOCKS];
     float scan_level_spread[NUNA_SCAN_LEVELS];
+    /* Streaming read rate of each SM on its own, GB/s: one block of 256 threads on that SM (every other SM
+     * idle) reads a 1 MiB L2-resident window four times with 16-byte L2-only loads.  Zero for SMs that did
+     * not report.                                                                                          */
+    float sm_read_gbs[NUNA_MAX_SMS];
 } nuna_topology_t;
 
 /* Measures, for every SM (indexed by %smid) and every buffer, the latency of dependent L2-only loads
  * to sampled lines of the caller's buffers (the analogue of the paper's per-compute-unit, per-address
  * remote-access sweep, Section 3.2), plus each SM's cold DRAM latency, clusters the SMs into domains
  * maps the home domain of a window of consecutive lines and of blocks of 4 KiB / 64 KiB / 2 MiB of buffer 0,
+ * measures each SM's solo streaming read rate,
  * and stores the result in *out and in the device context (where NUNA_PLACE_SM_LISTS plans read it).
  * bufs: HOST array of nbufs (<= NUNA_MAX_PROBE_BUFS) device pointers, bytes[b] >= 128 each, 16-byte
  * aligned.  One 8-byte word per sampled line (about 3000 lines at most) is overwritten during the measurement and restored

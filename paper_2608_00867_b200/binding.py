@@ -71,6 +71,7 @@ class NunaTopology(ctypes.Structure):
         ("scan_run_hist", ctypes.c_uint * NUNA_SCAN_RUN_BINS),
         ("scan_level_share", (ctypes.c_float * NUNA_SCAN_BLOCKS) * NUNA_SCAN_LEVELS),
         ("scan_level_spread", ctypes.c_float * NUNA_SCAN_LEVELS),
+        ("sm_read_gbs", ctypes.c_float * NUNA_MAX_SMS),
     ]
 
 

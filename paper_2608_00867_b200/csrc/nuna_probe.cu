@@ -114,6 +114,34 @@ __global__ void k_probe_miss(const unsigned char* base, const unsigned* starts, 
     ends[blockIdx.x] = (unsigned)idx;
 }
 
+// Solo streaming read rate of one SM: the block that lands on SM `target` reads the window `passes` times
+// with 16-byte L2-only loads (after one untimed pass that brings it into L2); every other block leaves at
+// once, so the measuring SM has the memory system to itself.  bytes / nanoseconds = GB/s.
+__global__ void k_probe_bw(const uint4* window, unsigned nvec, unsigned target, int passes, float* gbs, int max_sms)
+{
+    extern __shared__ unsigned char force_one_block_per_sm[];
+    __shared__ unsigned sink;
+    const unsigned s = read_smid();
+    if (s != target || (int)s >= max_sms) return;
+    unsigned acc = 0;
+    for (unsigned i = threadIdx.x; i < nvec; i += blockDim.x) acc ^= (unsigned)ld_cg_u64((unsigned long long)(window + i));
+    __syncthreads();
+    unsigned long long t0, t1;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0) :: "memory");
+    for (int p = 0; p < passes; ++p) {
+#pragma unroll 8
+        for (unsigned i = threadIdx.x; i < nvec; i += blockDim.x) {
+            unsigned x, y, z, w;
+            asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "l"(window + i) : "memory");
+            acc ^= x ^ y ^ z ^ w;
+        }
+    }
+    __syncthreads();
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1) :: "memory");
+    if (acc == 0x9E3779B9u) sink = acc;                            // keeps the loads alive
+    if (threadIdx.x == 0 && t1 > t0) gbs[s] = (float)((double)nvec * 16.0 * passes / (double)(t1 - t0));
+}
+
 static uint64_t splitmix(uint64_t& x)
 {
     uint64_t z = (x += 0x9E3779B97F4A7C15ull);
@@ -356,14 +384,14 @@ int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
     // ---- device scratch ---------------------------------------------------------------------------------
     unsigned long long** d_lines = nullptr;
     unsigned long long* d_saved = nullptr;
-    float *d_lat = nullptr, *d_miss = nullptr;
+    float *d_lat = nullptr, *d_miss = nullptr, *d_gbs = nullptr;
     int* d_seen = nullptr;
     unsigned *d_bad = nullptr, *d_next = nullptr, *d_starts = nullptr, *d_ends = nullptr;
     unsigned char *d_chain = nullptr, *d_flush = nullptr;
     const int nnodes = (int)std::max<size_t>(4096, std::min<size_t>(32768, c->l2_bytes / kNodeStride));
     const size_t flush_bytes = c->l2_bytes + (c->l2_bytes >> 2);
     const size_t smem_one_per_sm = 120 * 1024;
-    std::vector<float> lat0((size_t)max_sms * L), lat1((size_t)max_sms * L), miss(max_sms, 0.f);
+    std::vector<float> lat0((size_t)max_sms * L), lat1((size_t)max_sms * L), miss(max_sms, 0.f), gbs(max_sms, 0.f);
     std::vector<int> seen(max_sms, 0);
     std::vector<unsigned> next((size_t)nnodes), starts(c->num_sms), ends(c->num_sms, 0);
     unsigned bad = 0;
@@ -373,6 +401,7 @@ int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
     PROBE_CK(cudaMalloc(&d_saved, sizeof(unsigned long long) * L));
     PROBE_CK(cudaMalloc(&d_lat, sizeof(float) * (size_t)max_sms * L));
     PROBE_CK(cudaMalloc(&d_miss, sizeof(float) * max_sms));
+    PROBE_CK(cudaMalloc(&d_gbs, sizeof(float) * max_sms));
     PROBE_CK(cudaMalloc(&d_seen, sizeof(int) * max_sms));
     PROBE_CK(cudaMalloc(&d_bad, sizeof(unsigned)));
     PROBE_CK(cudaMalloc(&d_next, sizeof(unsigned) * nnodes));
@@ -382,6 +411,8 @@ int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
     PROBE_CK(cudaMalloc(&d_flush, flush_bytes));
     PROBE_CK(cudaFuncSetAttribute(k_probe_hit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_one_per_sm));
     PROBE_CK(cudaFuncSetAttribute(k_probe_miss, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_one_per_sm));
+    PROBE_CK(cudaFuncSetAttribute(k_probe_bw, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_one_per_sm));
+    PROBE_CK(cudaMemsetAsync(d_gbs, 0, sizeof(float) * max_sms, stream));
     PROBE_CK(cudaMemcpyAsync(d_lines, lines.data(), sizeof(void*) * L, cudaMemcpyHostToDevice, stream));
     PROBE_CK(cudaMemsetAsync(d_bad, 0, sizeof(unsigned), stream));
     PROBE_CK(cudaMemsetAsync(d_miss, 0, sizeof(float) * max_sms, stream));
@@ -417,6 +448,12 @@ int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
     k_flush<<<c->num_sms * 4, 256, 0, stream>>>(reinterpret_cast<uint4*>(d_flush), flush_bytes / 16);
     k_probe_miss<<<c->num_sms, 32, smem_one_per_sm, stream>>>(d_chain, d_starts, d_miss, d_ends, max_sms);
     g_launches.fetch_add(3, std::memory_order_relaxed);
+    // ---- solo streaming read rate, one SM after the other (the window is the start of the flush region) ---------
+    for (int s = 0; s < max_sms; ++s)
+        k_probe_bw<<<c->num_sms, 256, smem_one_per_sm, stream>>>(reinterpret_cast<const uint4*>(d_flush), 65536u, (unsigned)s, 4, d_gbs,
+                                                                  max_sms);
+    g_launches.fetch_add((unsigned long long)max_sms, std::memory_order_relaxed);
+    PROBE_CK(cudaMemcpyAsync(gbs.data(), d_gbs, sizeof(float) * max_sms, cudaMemcpyDeviceToHost, stream));
     PROBE_CK(cudaMemcpyAsync(miss.data(), d_miss, sizeof(float) * max_sms, cudaMemcpyDeviceToHost, stream));
     PROBE_CK(cudaMemcpyAsync(ends.data(), d_ends, sizeof(unsigned) * c->num_sms, cudaMemcpyDeviceToHost, stream));
     PROBE_CK(cudaMemcpyAsync(&bad, d_bad, sizeof(unsigned), cudaMemcpyDeviceToHost, stream));
@@ -430,6 +467,7 @@ int nuna_probe_topology(const void* const* bufs, const size_t* bytes, int nbufs,
             out->sm_reported[s] = seen[s] > 0;
             reported += seen[s] > 0;
             out->sm_lat_miss[s] = miss[s];
+            out->sm_read_gbs[s] = gbs[s];
         }
         out->sms_reported = reported;
         out->self_pointer_mismatches = (int)bad;
@@ -514,7 +552,7 @@ done:
         k_probe_words<<<(L + 127) / 128, 128, 0, stream>>>(d_lines, d_saved, L, 1);
         cudaStreamSynchronize(stream);
     }
-    cudaFree(d_lines); cudaFree(d_saved); cudaFree(d_lat); cudaFree(d_miss); cudaFree(d_seen); cudaFree(d_bad);
+    cudaFree(d_lines); cudaFree(d_saved); cudaFree(d_lat); cudaFree(d_miss); cudaFree(d_gbs); cudaFree(d_seen); cudaFree(d_bad);
     cudaFree(d_next); cudaFree(d_starts); cudaFree(d_ends); cudaFree(d_chain); cudaFree(d_flush);
     return status;
 }

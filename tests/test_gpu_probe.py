@@ -46,6 +46,14 @@ def test_latencies_are_physical(probed):
     assert 0.0 <= t.nonuniformity < 1.0
 
 
+def test_solo_read_rate_of_every_sm(probed):
+    _, _, t1, t2 = probed
+    a, b = np.array(t1.sm_read_gbs[:t1.num_sms]), np.array(t2.sm_read_gbs[:t2.num_sms])
+    assert (a > 10.0).all() and (a < 5000.0).all()              # every SM measured, physically plausible GB/s
+    assert np.median(np.abs(a - b) / a) < 0.10                  # the second probe agrees
+    assert a.max() / a.min() < 3.0                              # no SM is starved of bandwidth
+
+
 def test_repeatable_within_noise(probed):
     _, _, t1, t2 = probed
     a, b = np.array(t1.sm_lat_hit[:t1.num_sms]), np.array(t2.sm_lat_hit[:t2.num_sms])
