@@ -1,10 +1,17 @@
 // Device code of the emulated-rank collectives (sm_100a).
 //
-// All data movement is 16-byte vectorised and coalesced: one thread moves one
-// uint4 (8 bf16) per source per step, a warp covers 512 contiguous bytes of
-// every buffer it touches.  A thread first issues the loads of all N sources
-// (N independent 16-byte requests in flight per thread give the memory-level
-// parallelism), then folds them in rank order in binary32 and rounds once.
+// Two families of kernels.  Register kernels: all data movement is 16-byte
+// vectorised and coalesced, one thread moves one uint4 (8 bf16) per source per
+// step, a warp covers 512 contiguous bytes of every buffer it touches; a thread
+// first issues the loads of all N sources (N independent 16-byte requests in
+// flight per thread give the memory-level parallelism), then folds them in rank
+// order in binary32 and rounds once.  Bulk-copy kernels: one thread of a block
+// issues one-dimensional cp.async.bulk copies (plain form: this GPU's memory,
+// no multicast) that bring a tile's slices into shared memory and complete on an
+// mbarrier; the bytes in flight hold no registers, and pure copies (allgather,
+// alltoall) leave shared memory again by bulk stores.  Every wait in this file
+// (ready flag, barrier, copy completion) is bounded and ends in a latched status,
+// never in a trap or an endless spin.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
