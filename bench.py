@@ -95,18 +95,23 @@ def host_cores():
 
 
 def oracle_time(src, nthreads, seconds):
-    """The oracle as it stands, repeated for about `seconds` after a warm-up, in batches of 5 calls.
+    """The oracle as it stands, repeated for about `seconds` after a warm-up, in batches of 5 calls, writing into
+    destination arrays allocated once (with fresh arrays per call the loop times the allocator's page faults --
+    4 MiB per call -- and the result then swings by 2-3x from one process to the next with the state of its heap).
     Returns (best batch, median batch) in us per allreduce and the number of calls.  The best batch is the
     reported value: the host is shared, and interference only ever adds time."""
+    import numpy as np
+
     import oracle
+    out = [np.empty_like(a) for a in src]
     t_end = time.perf_counter() + min(0.5, seconds / 3)
     while time.perf_counter() < t_end:                           # thread pool, page faults, caches
-        oracle.allreduce(src, nthreads=nthreads)
+        oracle.allreduce(src, nthreads=nthreads, out=out)
     per, calls, t_stop = [], 0, time.perf_counter() + seconds
     while time.perf_counter() < t_stop or len(per) < 3:
         t0 = time.perf_counter()
         for _ in range(5):
-            oracle.allreduce(src, nthreads=nthreads)
+            oracle.allreduce(src, nthreads=nthreads, out=out)
         per.append((time.perf_counter() - t0) / 5 * 1e6)
         calls += 5
     per.sort()
@@ -218,15 +223,16 @@ def run_gpu(args):
     rep = Replicas(backend="nccl")
     rank, world, local = rep.rank, rep.world, rep.local
 
-    # first window of the CPU baseline, before any GPU work (rank 0 at N = 1 only)
-    cpu_early = None
-    if rank == 0 and world == 1:
-        cpu_early = oracle_time(workloads.make(workloads.config_decode_activation()), host_cores(), 2.0)
-
     peak_gbs, peak_src = measured_peaks()
     l2 = torch.cuda.get_device_properties(local).L2_cache_size
     num_sms = torch.cuda.get_device_properties(local).multi_processor_count
     nb.nuna_init(128 << 20)
+    # first window of the CPU baseline, before the GPU work starts (rank 0 at N = 1 only); the second one comes
+    # at the end
+    cpu_early = None
+    if rank == 0 and world == 1:
+        cpu_early = oracle_time(workloads.make(workloads.config_decode_activation()), host_cores(), 2.0)
+
     stream = torch.cuda.Stream()
     sampler = ClockSampler(local)
     if rank == 0:

@@ -86,12 +86,25 @@ def _check_src(src: Sequence[np.ndarray], length: int, storage=np.uint16):
             raise ValueError(f"every rank buffer must be a 1-D {np.dtype(storage).name} array of the same length")
 
 
-def allreduce(src: Sequence[np.ndarray], nthreads: int = 1, dtype: str = "bf16") -> List[np.ndarray]:
-    """One result array per destination rank (all equal by definition)."""
+def allreduce(src: Sequence[np.ndarray], nthreads: int = 1, dtype: str = "bf16",
+              out: Sequence[np.ndarray] = None) -> List[np.ndarray]:
+    """One result array per destination rank (all equal by definition).
+
+    ``out``: optional destination arrays to write into (one per rank, same shape and storage type as the
+    sources).  Without it fresh arrays are allocated on every call, and a timing of repeated calls then
+    measures the allocator's page faults as much as the fold."""
     n, count = len(src), len(src[0])
     _check_src(src, count, STORAGE[dtype])
     src = [np.ascontiguousarray(a) for a in src]
-    dst = [np.empty(count, dtype=STORAGE[dtype]) for _ in range(n)]
+    if out is None:
+        dst = [np.empty(count, dtype=STORAGE[dtype]) for _ in range(n)]
+    else:
+        if len(out) != n:
+            raise ValueError("need one destination per rank")
+        _check_src(out, count, STORAGE[dtype])
+        if not all(a.flags.c_contiguous and a.flags.writeable for a in out):
+            raise ValueError("destinations must be contiguous and writeable")
+        dst = list(out)
     getattr(_load(), f"nuna_oracle_allreduce_{dtype}")(_ptrs(src), _ptrs(dst), n, count, int(nthreads))
     return dst
 

@@ -282,3 +282,17 @@ def test_alltoall_of_replicated_blocks_is_allgather():
         assert np.array_equal(a2a[d], ag[d])
     assert np.array_equal(oracle.alltoall([shards[0]])[0], shards[0])   # one rank: identity
     assert np.array_equal(oracle.alltoall(src, 1)[2], oracle.alltoall(src, 8)[2])
+
+
+def test_allreduce_into_caller_owned_destinations():
+    """out=: same bits as the allocating form, written in place; bad destinations are refused."""
+    src = workloads.special_values(5, 1003, seed=77)
+    want = oracle.allreduce(src, nthreads=2)
+    out = [np.full(1003, 0xBEEF, dtype=np.uint16) for _ in range(5)]
+    got = oracle.allreduce(src, nthreads=2, out=out)
+    assert all(g is o for g, o in zip(got, out))
+    assert all(np.array_equal(o, w) for o, w in zip(out, want))
+    with pytest.raises(ValueError):
+        oracle.allreduce(src, out=out[:4])
+    with pytest.raises(ValueError):
+        oracle.allreduce(src, out=[np.zeros(1003, dtype=np.uint32) for _ in range(5)])
