@@ -73,7 +73,8 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
                                       allreduce distinguishes placements                                   */
 #define NUNA_PLACE_AUTO       2u   /* the placement-aware kernel measured fastest for the size (the co-located group
                                       that shares its tile through registers, NUNA_PLACE_REGS, from 1 MiB of
-                                      sources in total at 8 ranks or more, 2 MiB below), else exactly the
+                                      sources in total at 8 ranks or more, 2 MiB below; below that the group
+                                      sharing through L1 if NUNA_HINT_RESIDENT is set), else exactly the
                                       ROUNDROBIN kernel                                                    */
 #define NUNA_PLACE_MASK       3u
 /* `flags`, bit 4 (nuna_allreduce_twoshot only): the reducing block stores its tile straight into all N
