@@ -71,11 +71,11 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
                                       registers, shared memory, per-SM work lists or a cluster with
                                       NUNA_PLACE_REGS / _STAGED / _SM_LISTS / _CLUSTER; only the one-shot
                                       allreduce distinguishes placements                                   */
-#define NUNA_PLACE_AUTO       2u   /* the placement-aware kernel measured fastest for the size (the co-located group
-                                      that shares its tile through registers, NUNA_PLACE_REGS, from 1 MiB of
-                                      sources in total at 8 ranks or more, 2 MiB below; below that the group
-                                      sharing through L1 if NUNA_HINT_RESIDENT is set), else exactly the
-                                      ROUNDROBIN kernel                                                    */
+#define NUNA_PLACE_AUTO       2u   /* the placement-aware kernel measured fastest for the size and launch: the
+                                      co-located group that shares its tile through registers (NUNA_PLACE_REGS)
+                                      at every size with NUNA_LAUNCH_PDL or NUNA_HINT_RESIDENT, otherwise from
+                                      1 MiB of sources in total at 8 ranks or more, 2 MiB below; else exactly
+                                      the ROUNDROBIN kernel                                                */
 #define NUNA_PLACE_MASK       3u
 /* `flags`, bit 4 (nuna_allreduce_twoshot only): the reducing block stores its tile straight into all N
  * destinations, with no intermediate shard and no barrier.                                             */
@@ -88,7 +88,10 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 /* `flags`, bit 6: launch with programmatic stream serialization.  The kernel may be scheduled while its
  * predecessor in the stream drains; it waits for that grid's completion and memory visibility before
  * its first global access, so results are those of an ordinary stream-ordered launch.  The round-robin
- * one-shot ignores it above 16 MiB of sources, where it was measured not to pay.                         */
+ * one-shot ignores it above 16 MiB of sources, where it was measured not to pay.  Unless
+ * NUNA_HINT_RESIDENT is set, the register-sharing one-shot also asks L2, before that wait, to fetch each
+ * block's first tile of the sources (a prefetch returns nothing to the kernel; L2 is the point of
+ * coherence, so what the predecessor still writes is what the loads after the wait see).                */
 #define NUNA_LAUNCH_PDL       64u
 /* `flags`, bit 7, with NUNA_PLACE_AWARE on nuna_allreduce_oneshot: dispatch the co-located groups through
  * per-SM work lists.  The lists are planned by Algorithm 1 from the topology the last
@@ -273,10 +276,14 @@ int nuna_init(size_t scratch_bytes);
  *                           engine (one bulk load into shared memory, one bulk store per destination) by default (0,
  *                           tile size by message size); >= 8: tiles of that many 16-byte vectors; 1: the register
  *                           form instead (16-byte loads and stores by every thread)
+ *  NUNA_OPT_REGS_VECS       16-byte vectors per source per tile of the NUNA_PLACE_REGS kernel (8 ... 256; 0 = by size)
+ *  NUNA_OPT_PREFETCH        1: kernels launched with NUNA_LAUNCH_PDL do not ask L2 for their first tile ahead of the
+ *                           wait for their predecessor (0 = they do, unless NUNA_HINT_RESIDENT is given); a
+ *                           measurement aid, the prefetch changes no result
  * Returns NUNA_ERR_INVALID_ARG for an unknown option or a negative value.  Creates the context.          */
 enum { NUNA_OPT_BLOCKS = 0, NUNA_OPT_UNROLL = 1, NUNA_OPT_COLOC = 2, NUNA_OPT_AUTO_MIN_BYTES = 3, NUNA_OPT_TIMEOUT_MS = 4,
        NUNA_OPT_DOMAINS = 5, NUNA_OPT_STAGE_VECS = 6, NUNA_OPT_TWOSHOT_VECS = 7,
-       NUNA_OPT_AG_BULK_VECS = 8 };
+       NUNA_OPT_AG_BULK_VECS = 8, NUNA_OPT_REGS_VECS = 9, NUNA_OPT_PREFETCH = 10 };
 int nuna_set_option(int option, long long value);
 
 /* One-shot allreduce (Section 5.1, direct algorithm): every emulated rank d reads all N sources and

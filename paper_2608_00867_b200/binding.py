@@ -43,6 +43,7 @@ NUNA_HIST_BINS, NUNA_HIST_FIRST, NUNA_HIST_STEP = 48, 200, 4
 NUNA_SCAN_LINES, NUNA_SCAN_RUN_BINS, NUNA_SCAN_LEVELS, NUNA_SCAN_BLOCKS = 512, 16, 3, 8
 NUNA_OPT_BLOCKS, NUNA_OPT_UNROLL, NUNA_OPT_COLOC, NUNA_OPT_AUTO_MIN_BYTES, NUNA_OPT_TIMEOUT_MS = 0, 1, 2, 3, 4
 NUNA_OPT_DOMAINS, NUNA_OPT_STAGE_VECS, NUNA_OPT_TWOSHOT_VECS, NUNA_OPT_AG_BULK_VECS = 5, 6, 7, 8
+NUNA_OPT_REGS_VECS, NUNA_OPT_PREFETCH = 9, 10
 
 
 class NunaTopology(ctypes.Structure):

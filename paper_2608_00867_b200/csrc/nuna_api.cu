@@ -69,6 +69,8 @@ int get_context(Context** out)
         c->opt.twoshot_vecs = env_int("NUNA_TWOSHOT_VECS", 0);
         c->opt.keep_shard = env_int("NUNA_KEEP_SHARD", 0);
         c->opt.ag_bulk_vecs = env_int("NUNA_AG_BULK_VECS", 0);
+        c->opt.regs_vecs = env_int("NUNA_REGS_VECS", 0);
+        c->opt.prefetch = env_int("NUNA_PREFETCH", 0);
         g_ctx[dev] = c;
     }
     *out = g_ctx[dev];
@@ -291,26 +293,27 @@ static size_t ceil_div(size_t a, size_t b) { return (a + b - 1) / b; }
 // ---- collectives ---------------------------------------------------------------------------------
 
 // NUNA_PLACE_AUTO picks, per size, the one-shot kernel that was measured fastest on B200, never one that is
-// slower than the round-robin baseline: the co-located group that shares its tile through registers once the
-// message is large enough for the saved re-reads to matter (cold, 8 ranks: 256 KiB 2.14 vs 2.38 us, 512 KiB
-// 2.76 vs 3.30, 4 MiB 11.5 vs 15.1, 64 MiB 157 vs 225; L2-resident 512 KiB 1.72 vs 2.86; 16 ranks: 128 KiB
-// 2.33 vs 3.07, 4 MiB 21.5 vs 45.8), below that the round-robin kernel itself (8 ranks, 8 KiB: 1.51 vs 1.58 us).
-// The crossover was measured at 2, 3, 4, 8 and 16 ranks: 1 MiB of sources in total from 8 ranks up, 2 MiB below
-// (4 ranks: 256 KiB per rank 1.81 vs 1.79 us, 512 KiB 2.04 vs 2.11).  The other co-located forms (through L1,
-// through shared memory) are slower than this one at every size and stay opt-in.
+// slower than the round-robin baseline.  Measured at 2, 3, 4, 8 and 16 ranks, 8 KiB ... 4 MiB per rank
+// (us per graph node, 8 ranks; round-robin | group through L1 | group through registers):
+//   dependent launch, cold:      8 KiB 1.60 | 1.16 | 1.26   64 KiB 1.78 | 1.90 | 1.41   512 KiB 3.38 | 3.65 | 2.09   4 MiB 15.6 | 17.2 | 11.8
+//   dependent launch, resident:  8 KiB 1.18 | 1.16 | 1.05   64 KiB 1.21 | 1.19 | 1.09   512 KiB 2.99 | 2.48 | 1.64   4 MiB 15.1 | 17.1 | 10.5
+//   plain launch, resident:      8 KiB 1.58 | 1.55 | 1.53   64 KiB 1.62 | 1.59 | 1.58   512 KiB 3.41 | 2.88 | 2.15   4 MiB 15.1 | 17.1 | 11.2
+//   plain launch, cold:          8 KiB 2.02 | 1.56 | 2.00   64 KiB 2.16 | 2.46 | 2.27   512 KiB 3.78 | 4.24 | 3.29   4 MiB 15.5 | 17.2 | 12.5
+// The group that shares its tile through registers wins at every size behind a dependent launch and on
+// L2-resident sources; launched plainly on cold sources it wins from 1 MiB of sources in total (2 MiB below 8
+// ranks) and the round-robin kernel is kept below that.  The other co-located forms (through L1, through shared
+// memory) stay opt-in.
 enum class OneShotKernel { RoundRobin, Group, Staged, Regs };
 
 static OneShotKernel auto_kernel(const Context* c, const Options& o, int nranks, size_t bytes, unsigned flags)
 {
     (void)c;
     if (nranks < 2) return OneShotKernel::RoundRobin;
+    if (bytes < o.auto_min_bytes) return OneShotKernel::RoundRobin;
+    if (flags & (NUNA_LAUNCH_PDL | NUNA_HINT_RESIDENT)) return OneShotKernel::Regs;
     const size_t total = bytes * (size_t)nranks;
     const size_t from = nranks >= 8 ? ((size_t)1 << 20) : ((size_t)2 << 20);
-    if (total >= from && bytes >= o.auto_min_bytes) return OneShotKernel::Regs;
-    // below the crossover, sources the caller declares L2-resident are served a little faster by the group that
-    // shares its tile through L1 (8 ranks, warm: 8 KiB 1.08 vs 1.10 us, 64 KiB 1.16 vs 1.19 us; 160-node chain at
-    // 16 KiB 1.13 vs 1.17 us per node); cold it would lose (8 KiB: 2.02 vs 1.51 us), so only under the hint
-    return (flags & NUNA_HINT_RESIDENT) ? OneShotKernel::Group : OneShotKernel::RoundRobin;
+    return total >= from ? OneShotKernel::Regs : OneShotKernel::RoundRobin;
 }
 
 
@@ -511,15 +514,35 @@ static int launch_group(Context* c, const Options& o, const RankPtrs& p, size_t 
 }
 
 // Co-located group sharing the tile through registers: one (tile, C destinations) item per block.
+// Tile size (vectors per source), measured at 8 ranks, 8 KiB ... 64 MiB per rank, cold and L2-resident:
+// one block per SM with tiles of 8 ... 56 vectors while the message is that small (64 blocks of 8 vectors at
+// 8 KiB: 1.08 us per L2-resident graph node against 1.38 us with eight full blocks); then four blocks per SM
+// with tiles of 56 ... 256 vectors (512 KiB cold behind a dependent launch: 586 blocks of 56 vectors, 2.1 us
+// against 2.8 us with 256 full tiles); full tiles beyond.  Tiles never exceed a block's width: contiguous
+// chunks of several rows per block were slower from 8 MiB per rank (23.0 against 21.7 us).
+static unsigned regs_tile_vecs(const Context* c, const Options& o, size_t nvec, int ksplit)
+{
+    if (o.regs_vecs > 0) return (unsigned)std::min(kThreads, std::max(8, o.regs_vecs / 8 * 8));
+    const size_t units = nvec * (size_t)ksplit;
+    const size_t one = ceil_div(ceil_div(units, (size_t)c->num_sms), (size_t)8) * 8;
+    if (one <= 56) return (unsigned)std::max<size_t>(8, one);
+    const size_t four = ceil_div(ceil_div(units, (size_t)c->num_sms * 4), (size_t)8) * 8;
+    return (unsigned)std::min<size_t>(kThreads, std::max<size_t>(56, four));
+}
+
 template <int N, int C, int DT>
 static int launch_regs(Context* c, const Options& o, const RankPtrs& p, size_t count, unsigned flags, unsigned mode, cudaStream_t stream)
 {
     auto k = k_oneshot_regs<N, C, DT>;
+    constexpr int kSplit = (N + C - 1) / C;
     const size_t nvec = count / Elem<DT>::kElems;
-    const size_t ntiles = ceil_div(nvec, (size_t)kThreads);
-    const size_t nitems = std::max<size_t>(ntiles * ((N + C - 1) / C), (count % Elem<DT>::kElems) ? (size_t)N : 0);
+    const unsigned tv = regs_tile_vecs(c, o, nvec, kSplit);
+    const size_t ntiles = ceil_div(nvec, (size_t)tv);
+    const size_t nitems = std::max<size_t>(ntiles * kSplit, (count % Elem<DT>::kElems) ? (size_t)N : 0);
     const unsigned grid = pick_grid(c, o, std::max<size_t>(nitems, 1), NUNA_OCC(k), 0);
-    return launch(k, grid, stream, mode, p, count, ntiles, (flags & NUNA_HINT_RESIDENT) ? 0 : 1);
+    // cold sources behind a dependent launch: fetch into L2 while the predecessor drains
+    const bool prefetch = mode == kLaunchPdl && !(flags & NUNA_HINT_RESIDENT) && o.prefetch != 1;
+    return launch(k, grid, stream, mode, p, count, ntiles, tv, ((flags & NUNA_HINT_RESIDENT) ? 0 : 1) | (prefetch ? 2 : 0));
 }
 
 // Staged group kernel: one tile per block.  Tile size (vectors per source): large enough that a tile's
@@ -560,15 +583,13 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
     else if (place == NUNA_PLACE_AUTO) which = auto_kernel(c, o, nranks, bytes, flags);
     if (which == OneShotKernel::Regs) {
         const unsigned m = (flags & NUNA_LAUNCH_PDL) ? kLaunchPdl : kLaunchPlain;
-        // destinations per thread: half of them while the data comes from DRAM (two blocks per tile keep more loads
-        // in flight), all of them (eight at most) when it is L2-resident (one fetch per tile)
-        // (measured at 2-16 ranks: 16 ranks x 4 MiB cold 21.5 us with eight destinations per thread, 24.0 with four)
+        // destinations per thread: all of them (eight at most), so that a tile crosses the L2 -> SM fabric once;
+        // half of them for large cold messages, where two blocks per tile keep more DRAM loads in flight
+        // (8 ranks x 16 MiB cold: 41.8 us with four, 42.0 with eight; 16 ranks x 4 MiB: 21.5 us with eight, 24.0 with four)
         const int all = std::min(8, pow2_at_least(nranks));
-        int coloc = o.coloc > 0 ? o.coloc : ((flags & NUNA_HINT_RESIDENT) ? all : std::min(8, std::max(2, pow2_at_least(nranks) / 2)));
+        const bool large_cold = !(flags & NUNA_HINT_RESIDENT) && bytes >= ((size_t)8 << 20);
+        int coloc = o.coloc > 0 ? o.coloc : (large_cold ? std::min(8, std::max(2, pow2_at_least(nranks) / 2)) : all);
         while (coloc > 2 && coloc / 2 >= nranks) coloc >>= 1;
-        // a small message needs its blocks more than it needs the sharing: keep at least half a wave of them
-        const size_t tiles = ceil_div(nvec, (size_t)kThreads);
-        while (o.coloc <= 0 && coloc > 2 && tiles * ceil_div((size_t)nranks, (size_t)coloc) < (size_t)c->num_sms / 2) coloc >>= 1;
         return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
             constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
             if (coloc >= 8) return launch_regs<N, 8, DT>(c, o, p, count, flags, m, stream);
@@ -865,6 +886,8 @@ int nuna_set_option(int option, long long value)
         case NUNA_OPT_STAGE_VECS: c->opt.stage_vecs = (int)std::min<long long>(value, 4096); break;
         case NUNA_OPT_TWOSHOT_VECS: c->opt.twoshot_vecs = (int)std::min<long long>(value, 4096); break;
         case NUNA_OPT_AG_BULK_VECS: c->opt.ag_bulk_vecs = (int)std::min<long long>(value, 2048); break;
+        case NUNA_OPT_REGS_VECS: c->opt.regs_vecs = (int)std::min<long long>(value, kThreads); break;
+        case NUNA_OPT_PREFETCH: c->opt.prefetch = (int)std::min<long long>(value, 1); break;
         default: return NUNA_ERR_INVALID_ARG;
     }
     return NUNA_OK;

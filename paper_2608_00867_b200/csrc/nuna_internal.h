@@ -39,6 +39,8 @@ struct Options {
     int stage_vecs = 0;                  // NUNA_STAGE_VECS: vectors per source per tile of the staged one-shot (0 = by size)
     int twoshot_vecs = 0;                // NUNA_TWOSHOT_VECS: vectors per tile of the flag-synchronised two-shot (0 = by size)
     int ag_bulk_vecs = 0;                // NUNA_AG_BULK_VECS: > 0 = allgather through the bulk-copy engine with tiles of that many vectors
+    int regs_vecs = 0;                   // NUNA_REGS_VECS: vectors per tile of the register-sharing one-shot (0 = by size)
+    int prefetch = 0;                    // NUNA_PREFETCH: 1 = no L2 prefetch ahead of the dependent-launch wait
     int keep_shard = 0;                  // NUNA_KEEP_SHARD: do not discard consumed shard lines from L2 (measurement aid)
 };
 

@@ -55,6 +55,17 @@ __device__ __forceinline__ void pdl_trigger()
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Asks L2 to fetch `bytes` (a multiple of 16; 16-byte aligned address) of this GPU's memory.  Nothing is
+// returned to the thread and nothing is waited for, so it may be issued BEFORE pdl_wait(): L2 is the
+// point of coherence, a line the predecessor writes after the fetch is updated in place, and the loads
+// after the wait read the current data.  What it buys: the successor's blocks arrive while the
+// predecessor's last blocks drain and its writes are flushed; that window covers most of a DRAM round
+// trip, so cold sources are L2 hits by the time the wait returns.
+__device__ __forceinline__ void prefetch_l2_bulk(const void* g, unsigned bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(g), "r"(bytes) : "memory");
+}
+
 // ---- memory access helpers ----------------------------------------------------------------
 
 // Sources are read-only for the duration of a kernel and are re-read by other
@@ -454,19 +465,33 @@ __device__ __forceinline__ uint4 fold_vectors_own(const uint4 (&v)[N])
     return make_uint4(pack2<DT>(a[0], a[1]), pack2<DT>(a[2], a[3]), pack2<DT>(a[4], a[5]), pack2<DT>(a[6], a[7]));
 }
 
-// Work item = (tile of kThreads vectors, group of C destinations); one item per block.
+// Work item = (tile of `tv` <= kThreads vectors, group of C destinations); one item per block while the
+// grid allows.  The host sizes the tile by the message: a small message is cut into many small tiles
+// (every SM gets a few blocks of a few warps each; measured faster than few full blocks at every size
+// below 4 MiB per rank), a large one uses full tiles.
+// mode bit 0: streaming stores (destinations are not re-read soon); bit 1: every block asks L2 for its
+// first tile's source slices before it waits for the predecessor kernel (dependent launches with cold
+// sources only: without a predecessor there is nothing to overlap with).
 template <int N, int C, int DT>
 __global__ void __launch_bounds__(kThreads, min_blocks(N))
-k_oneshot_regs(const RankPtrs p, const size_t count, const size_t ntiles, const int stream_stores)
+k_oneshot_regs(const RankPtrs p, const size_t count, const size_t ntiles, const unsigned tv, const int mode)
 {
-    pdl_wait();
     constexpr int kSplit = (N + C - 1) / C;
     const size_t nvec = count / Elem<DT>::kElems;
     const size_t nitems = ntiles * kSplit;
+    if ((mode & 2) && blockIdx.x < nitems && threadIdx.x < N) {
+        const size_t i0 = ((size_t)blockIdx.x / kSplit) * tv;        // thread r fetches source r's slice
+        const uint4* a = p.src[0];
+#pragma unroll
+        for (int r = 1; r < N; ++r) if ((int)threadIdx.x == r) a = p.src[r];
+        if (i0 < nvec) prefetch_l2_bulk(a + i0, (unsigned)(nvec - i0 < (size_t)tv ? nvec - i0 : (size_t)tv) * 16u);
+    }
+    pdl_wait();
+    const int stream_stores = mode & 1;
     for (size_t item = blockIdx.x; item < nitems; item += gridDim.x) {
-        const size_t i = (item / kSplit) * kThreads + threadIdx.x;
+        const size_t i = (item / kSplit) * tv + threadIdx.x;
         const int d0 = (int)(item % kSplit) * C;
-        if (i < nvec) {
+        if (threadIdx.x < tv && i < nvec) {
             uint4 v[N];
 #pragma unroll
             for (int r = 0; r < N; ++r) v[r] = ld_src(p.src[r] + i);

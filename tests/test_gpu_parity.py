@@ -117,6 +117,58 @@ def test_staged_oneshot_tile_sizes(vecs):
     assert nb.nuna_device_status() == nb.NUNA_OK
 
 
+@pytest.mark.parametrize("vecs", [0, 8, 56, 104, 256])
+@pytest.mark.parametrize("n", [3, 8, 16])
+def test_register_oneshot_tile_sizes_and_prefetch(vecs, n):
+    """The register-sharing kernel at tile sizes from one line to a full block (0 = chosen by size), counts around
+    the tile edges and with a ragged tail, launched plainly, behind a dependent launch with the L2 prefetch ahead of
+    the wait, with the prefetch switched off, and with the resident hint (which also suppresses it): the prefetch
+    and the tile size change no bit."""
+    tv = vecs if vecs else 56
+    base = nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS
+    try:
+        nb.nuna_set_option(nb.NUNA_OPT_REGS_VECS, vecs)
+        for count in (8 * tv - 8, 8 * tv, 8 * tv + 8, 8 * tv * 5 + 3, 24 * 8192 + 1):
+            src = workloads.special_values(n, count, seed=7 * n + vecs + count % 101)
+            want = oracle.allreduce(src, nthreads=4)[0]
+            dsrc = upload(src)
+            for flags, no_prefetch in ((base, 0), (base | nb.NUNA_LAUNCH_PDL, 0), (base | nb.NUNA_LAUNCH_PDL, 1),
+                                       (base | nb.NUNA_LAUNCH_PDL | nb.NUNA_HINT_RESIDENT, 0)):
+                nb.nuna_set_option(nb.NUNA_OPT_PREFETCH, no_prefetch)
+                dst = Dst(n, count)
+                # two calls back to back: the second one's prefetch runs while the first is still writing
+                nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=flags)
+                nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=flags)
+                for got in dst.numpy():
+                    assert_same_bits(got, want, f"regs vecs={vecs} n={n} count={count} flags={flags} nopf={no_prefetch}")
+    finally:
+        nb.nuna_set_option(nb.NUNA_OPT_REGS_VECS, 0)
+        nb.nuna_set_option(nb.NUNA_OPT_PREFETCH, 0)
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
+def test_prefetch_ahead_of_the_wait_sees_the_predecessors_writes():
+    """A chain x -> allreduce -> allreduce -> ... in which every call's sources are the previous call's destinations,
+    launched back to back with dependent launches: each kernel's prefetch is issued while its predecessor is still
+    writing the very lines it asks for.  The values grow by a factor of N per node, so a stale line shows."""
+    n, count, nodes = 8, 64 * 1024, 5
+    src = [np.full(count, 0x3F80, dtype=np.uint16) for _ in range(n)]          # bf16 1.0
+    a, b = Dst(n, count), Dst(n, count)
+    flags = nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS | nb.NUNA_LAUNCH_PDL
+    for _ in range(20):
+        cur = upload(src)
+        for k in range(nodes):
+            out = a if k % 2 == 0 else b
+            nb.nuna_allreduce_oneshot(cur, out.view, count, flags=flags)
+            cur = out.view
+        got = out.numpy()
+        want = np.float32(n) ** nodes                                           # 8^5 = 32768, exact in bf16
+        for g in got:
+            vals = (g.astype(np.uint32) << 16).view(np.float32)
+            assert (vals == want).all()
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
 def test_config_small_two_ranks():
     w = workloads.config_small_oneshot()
     src = workloads.make(w)
