@@ -679,6 +679,16 @@ int launch_twoshot_flags(int num_sms, int blocks_override, const RankPtrs& p, in
 }
 
 // The put form: one tile per block by default; `max_blocks` > 0 makes it a grid-stride loop over that many blocks.
+// Whether a two-shot kernel asks L2 for its blocks' first tiles ahead of the dependent-launch wait: cold
+// device-memory sources, and a message small enough that the predecessor's drain is a visible share of it.
+// Measured with the put form (us, with | without): 8 ranks 2 MiB 6.16 | 6.44, 8 MiB 21.4 | 21.8, 16 MiB 42.1 | 42.1,
+// 64 MiB 162.5 | 160.8; 16 ranks 256 KiB 3.25 | 3.46, 1 MiB 6.74 | 6.59, 8 MiB 43.1 | 42.6; 4 ranks 32 MiB 41.3 | 41.7.
+static bool prefetch_pays(const Options& o, unsigned flags, int nranks, size_t bytes)
+{
+    if (!(flags & NUNA_LAUNCH_PDL) || (flags & NUNA_HINT_RESIDENT) || o.prefetch == 1) return false;
+    return bytes * (size_t)nranks <= (nranks <= 8 ? (size_t)128 << 20 : (size_t)8 << 20);
+}
+
 int launch_twoshot_put(Context* c, const RankPtrs& p, int nranks, int dtype, size_t count, unsigned flags, cudaStream_t stream,
                        unsigned max_blocks)
 {
@@ -691,7 +701,9 @@ int launch_twoshot_put(Context* c, const RankPtrs& p, int nranks, int dtype, siz
         const size_t ntiles = ceil_div(nvec, (size_t)kThreads * U);
         unsigned grid = pick_grid(c, o, std::max<size_t>(ntiles, 1), NUNA_OCC(k), 0);
         if (max_blocks > 0 && o.blocks <= 0) grid = std::min(grid, max_blocks);
-        return launch(k, grid, stream, mode, p, count, ntiles);
+        // device-memory sources behind a dependent launch: fetch the first tile into L2 while the predecessor drains
+        const bool prefetch = max_blocks == 0 && prefetch_pays(o, flags, nranks, count * elem_size(dtype));
+        return launch(k, grid, stream, mode, p, count, ntiles, prefetch ? 1 : 0);
     });
 }
 
@@ -708,7 +720,8 @@ int launch_twoshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
     }
     return launch_twoshot_flags(c->num_sms, o.blocks, p, nranks, dtype, count, (unsigned)std::max(0, o.twoshot_vecs), kMinFlagTileVec,
                                 scratch, tile_flags, c->bw, o.timeout_ns, (flags & NUNA_LAUNCH_PDL) != 0,
-                                (o.keep_shard ? 4u : 0u) | ((flags & NUNA_TWOSHOT_SYS_SCOPE) ? 8u : 0u), stream);
+                                (o.keep_shard ? 4u : 0u) | ((flags & NUNA_TWOSHOT_SYS_SCOPE) ? 8u : 0u) |
+                                    (prefetch_pays(o, flags, nranks, count * elem_size(dtype)) ? 16u : 0u), stream);
 }
 
 int launch_reduce_scatter(Context* c, const RankPtrs& p, int nranks, int dtype, size_t shard, unsigned flags,
@@ -937,9 +950,15 @@ int nuna_allreduce(const void* const* src, void* const* dst, int nranks, size_t 
     const size_t bytes = count * elem_size(dtype);
     size_t limit = nranks <= 2 ? ((size_t)1 << 20) : nranks <= 4 ? ((size_t)512 << 10)
                  : nranks <= 8 ? ((size_t)128 << 10) : ((size_t)64 << 10);
-    // with NUNA_PLACE_AUTO the one-shot side is the register-sharing kernel, which stays ahead of the put form
-    // up to 1 MiB per rank (8 ranks: 256 KiB 2.13 vs 2.28 us, 512 KiB 2.76 vs 2.83, 1 MiB 3.94 vs 3.96)
-    if ((flags & NUNA_PLACE_MASK) == NUNA_PLACE_AUTO) limit = std::max(limit, (size_t)1 << 20);
+    // with NUNA_PLACE_AUTO the one-shot side is the register-sharing kernel, which stays ahead of the put form up
+    // to 8 MiB of sources in total behind a dependent launch (8 ranks, cold: 128 KiB 1.51 vs 1.92 us, 1 MiB 3.33 vs
+    // 3.74, 2 MiB 6.44 vs 6.16; 4 ranks: 2 MiB 3.34 vs 3.52, 4 MiB 5.79 vs 5.73) and up to 2 MiB launched plainly
+    // (8 ranks: 256 KiB 2.65 vs 2.70, 512 KiB 3.29 vs 3.17); beyond 8 ranks, where it needs two passes over the
+    // sources, a quarter of that (16 ranks: 64 KiB 1.68 vs 2.69, 256 KiB 3.49 vs 3.25)
+    if ((flags & NUNA_PLACE_MASK) == NUNA_PLACE_AUTO) {
+        const size_t total = (flags & NUNA_LAUNCH_PDL) ? (size_t)8 << 20 : (size_t)2 << 20;
+        limit = std::max(limit, (nranks <= 8 ? total : total / 4) / (size_t)nranks);
+    }
     constexpr size_t kSyncFactor = 8;
     const bool sync_form = (flags & NUNA_TWOSHOT_SYNC) && !(flags & NUNA_TWOSHOT_PUT);
     const unsigned base = flags & ~(NUNA_TWOSHOT_SYNC | NUNA_TWOSHOT_PUT | (sync_form ? 0u : NUNA_TWOSHOT_SYS_SCOPE));

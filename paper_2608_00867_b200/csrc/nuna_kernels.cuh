@@ -1216,7 +1216,15 @@ k_twoshot_flags(const RankPtrs p, uint4* scratch, unsigned int* flags, const siz
     const size_t ntiles = nvec ? (nvec + tv - 1) / tv : 1;         // a ragged tail rides on the last tile
     const size_t lead = ntiles < lead_max ? ntiles : lead_max;
     if (threadIdx.x == 0) mbar_init(&bar, 1u);
-    pdl_wait();                                                     // before the first global access
+    if ((debug & 16u) && blockIdx.x < ntiles && threadIdx.x < N) {
+        // tickets come out nearly in block order: ask L2 for the tile this block will most likely produce
+        const size_t i0 = (size_t)blockIdx.x * tv;
+        const uint4* a = p.src[0];
+#pragma unroll
+        for (int r = 1; r < N; ++r) if ((int)threadIdx.x == r) a = p.src[r];
+        if (i0 < nvec) prefetch_l2_bulk(a + i0, (unsigned)(nvec - i0 < (size_t)tv ? nvec - i0 : (size_t)tv) * 16u);
+    }
+    pdl_wait();                                                     // before the first global load or store
     if (threadIdx.x == 0) {
         const unsigned long long t = atomicAdd(&bw->ticket, 1ull);  // epoch and ticket in one round trip
         if ((unsigned)t == gridDim.x - 1u)                          // the last ticket: set up the next launch
@@ -1299,10 +1307,17 @@ k_twoshot_flags(const RankPtrs p, uint4* scratch, unsigned int* flags, const siz
 // slower up to 4 MiB per rank -- 512 KiB: 3.2 vs 2.85 us -- and within 1.5 % beyond, so it was not kept.)
 template <int N, int U, int DT>
 __global__ void __launch_bounds__(kThreads, min_blocks(N * U))
-k_twoshot_put(const RankPtrs p, const size_t count, const size_t ntiles)
+k_twoshot_put(const RankPtrs p, const size_t count, const size_t ntiles, const int prefetch)
 {
-    pdl_wait();
     const size_t nvec = count / Elem<DT>::kElems;
+    if (prefetch && blockIdx.x < ntiles && threadIdx.x < N) {        // thread r: source r's slice of the first tile
+        const size_t i0 = (size_t)blockIdx.x * (size_t)(kThreads * U);
+        const uint4* a = p.src[0];
+#pragma unroll
+        for (int r = 1; r < N; ++r) if ((int)threadIdx.x == r) a = p.src[r];
+        if (i0 < nvec) prefetch_l2_bulk(a + i0, (unsigned)(nvec - i0 < (size_t)(kThreads * U) ? nvec - i0 : (size_t)(kThreads * U)) * 16u);
+    }
+    pdl_wait();
     for (size_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const size_t base = tile * (size_t)(kThreads * U) + threadIdx.x;
         uint4 v[U][N];

@@ -147,19 +147,23 @@ def test_register_oneshot_tile_sizes_and_prefetch(vecs, n):
     assert nb.nuna_device_status() == nb.NUNA_OK
 
 
-def test_prefetch_ahead_of_the_wait_sees_the_predecessors_writes():
+@pytest.mark.parametrize("algo", ["oneshot_regs", "twoshot_put", "twoshot_flags"])
+def test_prefetch_ahead_of_the_wait_sees_the_predecessors_writes(algo):
     """A chain x -> allreduce -> allreduce -> ... in which every call's sources are the previous call's destinations,
     launched back to back with dependent launches: each kernel's prefetch is issued while its predecessor is still
     writing the very lines it asks for.  The values grow by a factor of N per node, so a stale line shows."""
     n, count, nodes = 8, 64 * 1024, 5
     src = [np.full(count, 0x3F80, dtype=np.uint16) for _ in range(n)]          # bf16 1.0
     a, b = Dst(n, count), Dst(n, count)
-    flags = nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS | nb.NUNA_LAUNCH_PDL
+    call, flags = {"oneshot_regs": (nb.nuna_allreduce_oneshot, nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS),
+                   "twoshot_put": (nb.nuna_allreduce_twoshot, nb.NUNA_TWOSHOT_PUT),
+                   "twoshot_flags": (nb.nuna_allreduce_twoshot, 0)}[algo]
+    flags |= nb.NUNA_LAUNCH_PDL
     for _ in range(20):
         cur = upload(src)
         for k in range(nodes):
             out = a if k % 2 == 0 else b
-            nb.nuna_allreduce_oneshot(cur, out.view, count, flags=flags)
+            call(cur, out.view, count, flags=flags)
             cur = out.view
         got = out.numpy()
         want = np.float32(n) ** nodes                                           # 8^5 = 32768, exact in bf16
