@@ -531,7 +531,8 @@ static unsigned regs_tile_vecs(const Context* c, const Options& o, size_t nvec, 
 }
 
 template <int N, int C, int DT>
-static int launch_regs(Context* c, const Options& o, const RankPtrs& p, size_t count, unsigned flags, unsigned mode, cudaStream_t stream)
+static int launch_regs(Context* c, const Options& o, const RankPtrs& p, size_t count, unsigned flags, unsigned mode, bool may_prefetch,
+                       cudaStream_t stream)
 {
     auto k = k_oneshot_regs<N, C, DT>;
     constexpr int kSplit = (N + C - 1) / C;
@@ -541,7 +542,7 @@ static int launch_regs(Context* c, const Options& o, const RankPtrs& p, size_t c
     const size_t nitems = std::max<size_t>(ntiles * kSplit, (count % Elem<DT>::kElems) ? (size_t)N : 0);
     const unsigned grid = pick_grid(c, o, std::max<size_t>(nitems, 1), NUNA_OCC(k), 0);
     // cold sources behind a dependent launch: fetch into L2 while the predecessor drains
-    const bool prefetch = mode == kLaunchPdl && !(flags & NUNA_HINT_RESIDENT) && o.prefetch != 1;
+    const bool prefetch = may_prefetch && mode == kLaunchPdl && !(flags & NUNA_HINT_RESIDENT) && o.prefetch != 1;
     return launch(k, grid, stream, mode, p, count, ntiles, tv, ((flags & NUNA_HINT_RESIDENT) ? 0 : 1) | (prefetch ? 2 : 0));
 }
 
@@ -592,9 +593,11 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
         while (coloc > 2 && coloc / 2 >= nranks) coloc >>= 1;
         return dispatch(nranks, 1, dtype, [&](auto n_, auto, auto d_) -> int {
             constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
-            if (coloc >= 8) return launch_regs<N, 8, DT>(c, o, p, count, flags, m, stream);
-            if (coloc >= 4) return launch_regs<N, 4, DT>(c, o, p, count, flags, m, stream);
-            return launch_regs<N, 2, DT>(c, o, p, count, flags, m, stream);
+            // from 8 MiB per rank the prefetch only adds requests to a saturated memory system
+            // (8 ranks, four destinations per thread: 16 MiB 45.5 us with, 41.2 without; 64 MiB 175 against 158)
+            if (coloc >= 8) return launch_regs<N, 8, DT>(c, o, p, count, flags, m, !large_cold, stream);
+            if (coloc >= 4) return launch_regs<N, 4, DT>(c, o, p, count, flags, m, !large_cold, stream);
+            return launch_regs<N, 2, DT>(c, o, p, count, flags, m, !large_cold, stream);
         });
     }
     if (which == OneShotKernel::Staged) {
@@ -955,14 +958,18 @@ int nuna_allreduce(const void* const* src, void* const* dst, int nranks, size_t 
     // 3.74, 2 MiB 6.44 vs 6.16; 4 ranks: 2 MiB 3.34 vs 3.52, 4 MiB 5.79 vs 5.73) and up to 2 MiB launched plainly
     // (8 ranks: 256 KiB 2.65 vs 2.70, 512 KiB 3.29 vs 3.17); beyond 8 ranks, where it needs two passes over the
     // sources, a quarter of that (16 ranks: 64 KiB 1.68 vs 2.69, 256 KiB 3.49 vs 3.25)
+    // From 8 MiB per rank at 8 ranks or fewer it is ahead again, with two blocks per tile (8 ranks: 8 MiB 21.3 vs 21.6 us,
+    // 16 MiB 41.2 vs 42.1, 64 MiB 157.7 vs 160.8).
+    bool oneshot_large = false;
     if ((flags & NUNA_PLACE_MASK) == NUNA_PLACE_AUTO) {
         const size_t total = (flags & NUNA_LAUNCH_PDL) ? (size_t)8 << 20 : (size_t)2 << 20;
         limit = std::max(limit, (nranks <= 8 ? total : total / 4) / (size_t)nranks);
+        oneshot_large = nranks <= 8 && bytes >= ((size_t)8 << 20) && !(flags & NUNA_HINT_RESIDENT);
     }
     constexpr size_t kSyncFactor = 8;
     const bool sync_form = (flags & NUNA_TWOSHOT_SYNC) && !(flags & NUNA_TWOSHOT_PUT);
     const unsigned base = flags & ~(NUNA_TWOSHOT_SYNC | NUNA_TWOSHOT_PUT | (sync_form ? 0u : NUNA_TWOSHOT_SYS_SCOPE));
-    if (nranks <= 1 || bytes <= (sync_form ? limit * kSyncFactor : limit))
+    if (nranks <= 1 || bytes <= (sync_form ? limit * kSyncFactor : limit) || (oneshot_large && !sync_form))
         return nuna_allreduce_oneshot(src, dst, nranks, count, dtype, base, stream);
     return nuna_allreduce_twoshot(src, dst, nranks, count, dtype, sync_form ? base : (base | NUNA_TWOSHOT_PUT), stream);
 }
