@@ -773,7 +773,7 @@ int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard_byt
         if (tiles * (size_t)nranks <= ((size_t)1 << 24)) {
             t_dyn_smem = tv * 16u;
             return launch(k_allgather_bulk, (unsigned)(tiles * nranks), stream, mode, p, nranks, shard_vec, tiles, tv, &c->bw->status,
-                          o.timeout_ns);
+                          o.timeout_ns, prefetch_pays(o, flags, nranks, shard_vec * 16) ? 1 : 0);
         }
     }
     // One block per (rank, tile) storing to all N destinations.  Splitting a tile's destinations over
@@ -805,7 +805,8 @@ int launch_alltoall(Context* c, const RankPtrs& p, int nranks, size_t block_byte
         const size_t grid = tiles * (size_t)nranks * (size_t)nranks;
         if (grid <= ((size_t)1 << 24)) {
             t_dyn_smem = tv * 16u;
-            return launch(k_alltoall_bulk, (unsigned)grid, stream, mode, p, nranks, block_vec, tiles, tv, &c->bw->status, o.timeout_ns);
+            return launch(k_alltoall_bulk, (unsigned)grid, stream, mode, p, nranks, block_vec, tiles, tv, &c->bw->status, o.timeout_ns,
+                          prefetch_pays(o, flags, nranks, block_vec * 16 * (size_t)nranks) ? 1 : 0);
         }
     }
     constexpr int U = 2;

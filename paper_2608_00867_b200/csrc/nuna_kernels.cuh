@@ -872,6 +872,9 @@ __device__ __forceinline__ void reduce_tile(const RankPtrs& p, uint4* out, size_
     }
 }
 
+// (No L2 prefetch ahead of the dependent-launch wait here: this kernel reads N bytes for every byte it writes and is
+// bound by the reads at every size, so the extra requests only cost -- 8 x 512 KiB 2.43 against 2.16 us, 8 x 4 MiB 7.27
+// against 6.40.)
 template <int N, int U, int DT>
 __global__ void __launch_bounds__(kThreads, min_blocks(N * U))
 k_reduce_scatter(const RankPtrs p, const size_t shard_vec, const size_t tiles_per_shard)
@@ -961,7 +964,7 @@ __device__ __forceinline__ void bulk_store_drain()       // this thread's bulk s
 // tv = vectors per tile; shared memory = tv * 16 bytes.
 __global__ void __launch_bounds__(kThreads)
 k_allgather_bulk(const RankPtrs p, const int nranks, const size_t shard_vec, const size_t tiles_per_shard, const unsigned tv,
-                 unsigned* status, const unsigned long long timeout_ns)
+                 unsigned* status, const unsigned long long timeout_ns, const int prefetch)
 {
     extern __shared__ __align__(128) unsigned char stage_raw[];
     __shared__ __align__(8) uint64_t bar;
@@ -969,7 +972,10 @@ k_allgather_bulk(const RankPtrs p, const int nranks, const size_t shard_vec, con
     const size_t tile = blockIdx.x / (unsigned)nranks;
     const size_t base = tile * tv;
     const unsigned nv = (tile < tiles_per_shard && base < shard_vec) ? (unsigned)((shard_vec - base < tv) ? shard_vec - base : tv) : 0u;
-    if (threadIdx.x == 0) mbar_init(&bar, 1u);
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1u);
+        if (prefetch && nv != 0u) prefetch_l2_bulk(p.src[r] + base, nv * 16u);     // ahead of the wait: see prefetch_l2_bulk
+    }
     __syncthreads();
     pdl_wait();
     if (nv != 0u && threadIdx.x < (unsigned)nranks) {
@@ -1033,7 +1039,7 @@ k_alltoall(const RankPtrs p, const int nranks, const size_t block_vec, const siz
 // touching a register.  tv = vectors per tile; shared memory = tv * 16 bytes; one block per (pair, tile).
 __global__ void __launch_bounds__(kThreads)
 k_alltoall_bulk(const RankPtrs p, const int nranks, const size_t block_vec, const size_t tiles_per_block, const unsigned tv,
-                unsigned* status, const unsigned long long timeout_ns)
+                unsigned* status, const unsigned long long timeout_ns, const int prefetch)
 {
     extern __shared__ __align__(128) unsigned char stage_raw[];
     __shared__ __align__(8) uint64_t bar;
@@ -1044,6 +1050,7 @@ k_alltoall_bulk(const RankPtrs p, const int nranks, const size_t block_vec, cons
     const unsigned nv = (tile < tiles_per_block && base < block_vec) ? (unsigned)((block_vec - base < tv) ? block_vec - base : tv) : 0u;
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1u);
+        if (prefetch && nv != 0u) prefetch_l2_bulk(p.src[r] + (size_t)d * block_vec + base, nv * 16u);
         pdl_wait();
         if (nv != 0u) {
             mbar_expect_tx(&bar, nv * 16u);
