@@ -476,11 +476,36 @@ def run_gpu(args):
                           "cold": lat_summary(sum(nb.debug_access_latency(*sets[1 + i], count, pl) for i in range(len(sets) - 1)))}
         emit("first_load_latency_512KiB", lat)
 
+        c1 = (1 << 20) // 2
+        isets = make_sets(N_RANKS, c1, c1, 0, "normal", 77, max_sets=2)
+        # ---- sensitivity to the number of thread blocks and of SM domains (Section 6.5) ------------------------
+        # (Runs before the section with background load: timed right after its burst of dense GEMMs these
+        # latency-bound kernels read 30-50 % slower than in a fresh process, 140-180 against 95 us at 8 blocks.)
+        blocks_rows = {}
+        for label, fn_of in (("oneshot_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c1, stream=st))),
+                             ("twoshot_put_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c1, flags=nb.NUNA_TWOSHOT_PUT, stream=st)))):
+            row = {}
+            for blocks in (8, 37, 148, 592, 0):
+                nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, blocks)
+                row["default" if blocks == 0 else str(blocks)] = round(per_call_us(fn_of(), isets, 200), 3)
+            nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, 0)
+            blocks_rows[label] = row
+        emit("blocks_sensitivity_resident_us", blocks_rows)
+        if True:
+            dom_rows = {}
+            sm_flags = nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS
+            for label, cnt, ss in (("512KiB", count, sets[:1]), ("1MiB", c1, isets[:1])):
+                row = {}
+                for D in (1, 2, 4, 8):
+                    nb.nuna_set_option(nb.NUNA_OPT_DOMAINS, D)
+                    fn = lambda s, d, st, c=cnt: nb.nuna_allreduce_oneshot(s, d, c, flags=sm_flags, stream=st)
+                    row[str(D)] = round(per_call_us(fn, ss, 200), 3)
+                nb.nuna_set_option(nb.NUNA_OPT_DOMAINS, 0)
+                dom_rows[label] = row
+            emit("domain_count_sensitivity_sm_lists_resident_us", dom_rows)
         # ---- robustness to concurrent work (the paper runs its collectives beside a GEMM, Section 6.6) ------------
         # 1 MiB per rank one-shot, L2-resident sources, while a second stream runs (a) nothing, (b) a streaming
         # copy, (c) a dense bf16 matmul (a library GEMM used only as a load generator).
-        c1 = (1 << 20) // 2
-        isets = make_sets(N_RANKS, c1, c1, 0, "normal", 77, max_sets=2)
         side = torch.cuda.Stream()
         big_a = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         big_b = torch.empty_like(big_a)
@@ -514,29 +539,7 @@ def run_gpu(args):
             inter[lname] = row
         emit("interference_1MiB_resident", inter)
 
-        # ---- sensitivity to the number of thread blocks and of SM domains (Section 6.5) ------------------------
-        blocks_rows = {}
-        for label, fn_of in (("oneshot_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c1, stream=st))),
-                             ("twoshot_put_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c1, flags=nb.NUNA_TWOSHOT_PUT, stream=st)))):
-            row = {}
-            for blocks in (8, 37, 148, 592, 0):
-                nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, blocks)
-                row["default" if blocks == 0 else str(blocks)] = round(per_call_us(fn_of(), isets, 200), 3)
-            nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, 0)
-            blocks_rows[label] = row
-        emit("blocks_sensitivity_resident_us", blocks_rows)
-        if True:
-            dom_rows = {}
-            sm_flags = nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_SM_LISTS
-            for label, cnt, ss in (("512KiB", count, sets[:1]), ("1MiB", c1, isets[:1])):
-                row = {}
-                for D in (1, 2, 4, 8):
-                    nb.nuna_set_option(nb.NUNA_OPT_DOMAINS, D)
-                    fn = lambda s, d, st, c=cnt: nb.nuna_allreduce_oneshot(s, d, c, flags=sm_flags, stream=st)
-                    row[str(D)] = round(per_call_us(fn, ss, 200), 3)
-                nb.nuna_set_option(nb.NUNA_OPT_DOMAINS, 0)
-                dom_rows[label] = row
-            emit("domain_count_sensitivity_sm_lists_resident_us", dom_rows)
+        time.sleep(0.3)                                  # idle gap between the background load and the sweep
         del isets, big_a, big_b, ma, mb
         torch.cuda.empty_cache()
 
@@ -545,6 +548,7 @@ def run_gpu(args):
         algos = {
             "oneshot": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, stream=st)),
             "oneshot_aware": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=nb.NUNA_PLACE_AWARE, stream=st)),
+            "oneshot_auto": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c, flags=nb.NUNA_PLACE_AUTO, stream=st)),
             "oneshot_regs_pdl": lambda c: (lambda s, d, st: nb.nuna_allreduce_oneshot(
                 s, d, c, flags=P | nb.NUNA_PLACE_AWARE | nb.NUNA_PLACE_REGS, stream=st)),
             "twoshot": lambda c: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c, stream=st)),
@@ -580,6 +584,7 @@ def run_gpu(args):
             row["isolated_twoshot_us"] = isolated_stats(algos["twoshot"](c), ssets, 200 if B <= (4 << 20) else 40)
             row["isolated_twoshot_put_us"] = isolated_stats(algos["twoshot_put"](c), ssets, 200 if B <= (4 << 20) else 40)
             row["isolated_oneshot_warm_us"] = isolated_stats(algos["oneshot"](c), ssets[:1], 100 if B <= (4 << 20) else 20)
+            row["isolated_selected_us"] = isolated_stats(algos["selected_pdl"](c), ssets, 200 if B <= (4 << 20) else 40)
             best = min(algos, key=lambda a: row[a]["cold_us"])
             row["best"] = best
             row["best_frac_of_peak"] = row[best]["cold_frac_of_peak"]

@@ -658,7 +658,7 @@ int launch_twoshot_flags(int num_sms, int blocks_override, const RankPtrs& p, in
         // wave's consumers wait (10.3 us against 7.6 us with 12 KiB tiles), hence the step back there.
         const size_t src_bytes = bytes * (size_t)nranks;
         const unsigned tile_src = src_bytes <= ((size_t)512 << 10) ? 4096u : src_bytes <= ((size_t)1 << 20) ? 8192u
-                                : src_bytes <= ((size_t)4 << 20) ? 16384u : src_bytes <= ((size_t)8 << 20) ? 12288u
+                                : src_bytes <= ((size_t)8 << 20) ? 12288u
                                 : src_bytes <= ((size_t)32 << 20) ? 16384u : 32768u;
         tv = tile_src / 16u / (unsigned)nranks;
     }
