@@ -82,16 +82,18 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
 #define NUNA_TWOSHOT_PUT      16u
 /* `flags`, bit 5: hint that the sources were just written and are L2-resident (the decode case: a GEMM
  * epilogue produced them).  The register-sharing and shared-memory-staged one-shot kernels then co-locate
- * all destinations of a tile (one fetch per tile) and store with the ordinary cache policy instead of
- * evict-first.                                                                                          */
+ * all destinations of a tile (one fetch per tile) at every size, store with the ordinary cache policy
+ * instead of evict-first, and no kernel prefetches ahead of a dependent launch's wait.                  */
 #define NUNA_HINT_RESIDENT    32u
 /* `flags`, bit 6: launch with programmatic stream serialization.  The kernel may be scheduled while its
  * predecessor in the stream drains; it waits for that grid's completion and memory visibility before
  * its first global access, so results are those of an ordinary stream-ordered launch.  The round-robin
  * one-shot ignores it above 16 MiB of sources, where it was measured not to pay.  Unless
- * NUNA_HINT_RESIDENT is set, the register-sharing one-shot also asks L2, before that wait, to fetch each
- * block's first tile of the sources (a prefetch returns nothing to the kernel; L2 is the point of
- * coherence, so what the predecessor still writes is what the loads after the wait see).                */
+ * NUNA_HINT_RESIDENT is set, a block of the register-sharing one-shot (below 8 MiB per rank), of either
+ * two-shot form (up to 128 MiB of sources; 8 MiB beyond 8 ranks) and of the bulk-copy allgather and
+ * alltoall also asks L2, before that wait, to fetch its first tile of the sources (a prefetch returns
+ * nothing to the kernel; L2 is the point of coherence, so what the predecessor still writes is what the
+ * loads after the wait see).                                                                            */
 #define NUNA_LAUNCH_PDL       64u
 /* `flags`, bit 7, with NUNA_PLACE_AWARE on nuna_allreduce_oneshot: dispatch the co-located groups through
  * per-SM work lists.  The lists are planned by Algorithm 1 from the topology the last
