@@ -359,6 +359,40 @@ def test_graph_replay_gives_same_bits():
             assert np.array_equal(t.cpu().numpy().view(np.uint16), want)
 
 
+def test_headline_launch_configuration_matches_oracle():
+    """The configuration the benchmark times: 8 x 512 KiB, placement AUTO with dependent launches, as nodes of one
+    CUDA graph rotating over buffer sets (distinct data in each), replayed.  Every destination of every set is
+    compared with the oracle after each replay, so a prefetch or a dependent launch that ran ahead of its data would show."""
+    w = workloads.config_decode_activation()
+    nsets, passes = 6, 3
+    srcs = [workloads.rank_buffers(w.nranks, w.count, "normal", seed=500 + k) for k in range(nsets)]
+    want = [oracle.allreduce(x, nthreads=4)[0] for x in srcs]
+    dsrc = [upload(x) for x in srcs]
+    ddst = [[torch.zeros(w.count, dtype=torch.int16, device="cuda") for _ in range(w.nranks)] for _ in range(nsets)]
+    flags = nb.NUNA_PLACE_AUTO | nb.NUNA_LAUNCH_PDL
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        nb.nuna_allreduce_oneshot(dsrc[0], ddst[0], w.count, flags=flags, stream=s)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=s):
+            for _ in range(passes):
+                for k in range(nsets):
+                    nb.nuna_allreduce_oneshot(dsrc[k], ddst[k], w.count, flags=flags, stream=s)
+    for _ in range(3):
+        for dset in ddst:
+            for t in dset:
+                t.zero_()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(s):
+            g.replay()
+        torch.cuda.synchronize()
+        for k in range(nsets):
+            for t in ddst[k]:
+                assert np.array_equal(t.cpu().numpy().view(np.uint16), want[k]), f"set {k}"
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
 @pytest.mark.parametrize("flags", [0, nb.NUNA_LAUNCH_PDL, nb.NUNA_LAUNCH_PDL | nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT,
                                    nb.NUNA_CHAIN_GRAPH, nb.NUNA_CHAIN_PERSISTENT])
 @pytest.mark.parametrize("two_shot", [False, True])
