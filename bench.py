@@ -476,6 +476,46 @@ def run_gpu(args):
                           "cold": lat_summary(sum(nb.debug_access_latency(*sets[1 + i], count, pl) for i in range(len(sets) - 1)))}
         emit("first_load_latency_512KiB", lat)
 
+        # ---- where the time between two dependent launches goes (512 KiB one-shot, the headline kernel) -----------
+        # A graph of traced launches: thread 0 of every block records when the block started, when its wait for
+        # the predecessor returned and when it had issued its last store (global-timer ns), and its SM.
+        def timeline(tsets, tflags, no_prefetch):
+            nodes, TB = 200, nb.DEBUG_TRACE_BLOCKS
+            nb.nuna_set_option(nb.NUNA_OPT_PREFETCH, 1 if no_prefetch else 0)
+            trace = torch.zeros(nodes * TB * 4, dtype=torch.int64, device="cuda")
+            grid = [0]
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(stream):
+                grid[0] = nb.debug_oneshot_regs_traced(*tsets[0], count, tflags, 0, trace, stream)
+                torch.cuda.synchronize()
+                with torch.cuda.graph(g, stream=stream):
+                    for i in range(nodes):
+                        nb.debug_oneshot_regs_traced(*tsets[i % len(tsets)], count, tflags, i, trace, stream)
+                for _ in range(3):
+                    g.replay()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                g.replay()
+                e1.record(stream)
+                torch.cuda.synchronize()
+            nb.nuna_set_option(nb.NUNA_OPT_PREFETCH, 0)
+            t = trace.cpu().numpy().reshape(nodes, TB, 4)[20:, :min(grid[0], TB)].astype(np.int64)
+            start, release, end = np.median(t[:, :, 0], axis=1), t[:, :, 1].min(axis=1), t[:, :, 2].max(axis=1)
+            per_sm = [np.bincount(row[:, 3]) for row in t]
+            med = lambda a: round(float(np.median(a)) / 1e3, 3)
+            return {"grid_blocks": grid[0], "per_node_us_traced": round(e0.elapsed_time(e1) * 1e3 / nodes, 3),
+                    "blocks_resident_before_release_us": med(release - start),
+                    "release_to_last_store_us": med(end - release),
+                    "last_store_to_next_release_us": med(release[1:] - end[:-1]),
+                    "release_to_release_us": med(np.diff(release)),
+                    "sms_used_median": int(np.median([(b > 0).sum() for b in per_sm])),
+                    "max_blocks_per_sm": int(max(b.max() for b in per_sm)), "timer_resolution_ns": 32}
+        P0 = nb.NUNA_LAUNCH_PDL
+        emit("dependent_launch_timeline_512KiB", {
+            "cold_prefetch": timeline(sets, P0, False), "cold_no_prefetch": timeline(sets, P0, True),
+            "l2_resident": timeline(sets[:2], P0 | nb.NUNA_HINT_RESIDENT, False),
+            "plain_launch_cold": timeline(sets, 0, False)})
+
         c1 = (1 << 20) // 2
         isets = make_sets(N_RANKS, c1, c1, 0, "normal", 77, max_sets=2)
         # ---- sensitivity to the number of thread blocks and of SM domains (Section 6.5) ------------------------

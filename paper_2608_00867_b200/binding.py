@@ -157,6 +157,9 @@ def lib() -> ctypes.CDLL:
         L.nuna_debug_barrier_selftest.restype = ctypes.c_int
         L.nuna_debug_access_latency.argtypes = [vpp, vpp, ctypes.c_size_t, ctypes.c_int, ctypes.POINTER(ctypes.c_uint)]
         L.nuna_debug_access_latency.restype = ctypes.c_int
+        L.nuna_debug_oneshot_regs_traced.argtypes = [vpp, vpp, ctypes.c_size_t, ctypes.c_uint, ctypes.c_uint, ctypes.c_void_p,
+                                                     ctypes.POINTER(ctypes.c_uint), ctypes.c_void_p]
+        L.nuna_debug_oneshot_regs_traced.restype = ctypes.c_int
         L.nuna_debug_twoshot.argtypes = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint, ctypes.c_uint]
         L.nuna_debug_twoshot.restype = ctypes.c_int
         _lib = L
@@ -394,6 +397,21 @@ def debug_access_latency(src, dst, count, placement: int, launches: int = 1):
         if st != NUNA_OK:
             raise NunaError(st, "nuna_debug_access_latency")
     return hist
+
+
+DEBUG_TRACE_BLOCKS = 1024
+
+
+def debug_oneshot_regs_traced(src, dst, count, flags: int, slot: int, trace, stream=None) -> int:
+    """One traced launch of the register-sharing one-shot (8 ranks, bf16): thread 0 of block b writes its start,
+    wait-return and end times (global-timer ns) and its SM to ``trace`` (a device int64 tensor viewed as
+    [slots][DEBUG_TRACE_BLOCKS][4]) at ``slot``.  Capturable.  Returns the grid size."""
+    grid = ctypes.c_uint(0)
+    st = lib().nuna_debug_oneshot_regs_traced(ptr_table(src), ptr_table(dst), count, flags, slot,
+                                              ctypes.c_void_p(_addr(trace)), ctypes.byref(grid), _stream(stream))
+    if st != NUNA_OK:
+        raise NunaError(st, "nuna_debug_oneshot_regs_traced")
+    return grid.value
 
 
 def debug_twoshot(src, dst, count, dtype=NUNA_BF16, timeout_ms: int = 1000, unset_flags: bool = False) -> int:

@@ -1247,6 +1247,31 @@ int nuna_debug_access_latency(const void* const* src, void* const* dst, size_t c
     return st;
 }
 
+// See nuna_debug.h.  The same tile size, grid and mode bits as launch_regs<8, 8, bf16>.
+int nuna_debug_oneshot_regs_traced(const void* const* src, void* const* dst, size_t count, unsigned flags, unsigned slot,
+                                   unsigned long long* trace, unsigned* grid_blocks, void* stream)
+{
+    constexpr int N = 8;
+    int st = check_args(src, dst, N, count, count, NUNA_BF16, flags & (NUNA_LAUNCH_PDL | NUNA_HINT_RESIDENT), true);
+    if (st != NUNA_OK) return st;
+    if (!trace || count == 0 || (flags & ~(NUNA_LAUNCH_PDL | NUNA_HINT_RESIDENT)) != 0u) return NUNA_ERR_INVALID_ARG;
+    Context* c = nullptr;
+    if ((st = get_context(&c)) != NUNA_OK) return st;
+    const Options o = snapshot(c);
+    auto k = k_oneshot_regs_timed<N, 8, kBf16>;
+    const size_t nvec = count / 8;
+    const unsigned tv = regs_tile_vecs(c, o, nvec, 1);
+    const size_t ntiles = ceil_div(nvec, (size_t)tv);
+    const size_t nitems = std::max<size_t>(ntiles, (count % 8) ? (size_t)N : 0);
+    const unsigned grid = pick_grid(c, o, std::max<size_t>(nitems, 1), NUNA_OCC(k), 0);
+    const unsigned mode = (flags & NUNA_LAUNCH_PDL) ? kLaunchPdl : kLaunchPlain;
+    const bool large_cold = !(flags & NUNA_HINT_RESIDENT) && count * 2 >= ((size_t)8 << 20);
+    const bool prefetch = !large_cold && mode == kLaunchPdl && !(flags & NUNA_HINT_RESIDENT) && o.prefetch != 1;
+    if (grid_blocks) *grid_blocks = grid;
+    return launch(k, grid, (cudaStream_t)stream, mode, make_ptrs(src, dst, N), count, ntiles, tv,
+                  ((flags & NUNA_HINT_RESIDENT) ? 0 : 1) | (prefetch ? 2 : 0), trace, slot, (unsigned)NUNA_DEBUG_TRACE_BLOCKS);
+}
+
 /* Test hook: a flag-synchronised two-shot whose consumers wait for a flag value that nobody publishes
  * (debug_bits = 1): every consumer wait runs out after timeout_ms, the kernel returns, destinations stay
  * unwritten and the status word latches NUNA_ERR_TIMEOUT; nothing traps or hangs.  debug_bits = 0 is the

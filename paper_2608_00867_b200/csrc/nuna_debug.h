@@ -39,6 +39,17 @@ int nuna_debug_twoshot(const void* const* src, void* const* dst, int nranks, siz
 #define NUNA_DEBUG_LAT_STEP 32
 int nuna_debug_access_latency(const void* const* src, void* const* dst, size_t count, int placement, unsigned* hist);
 
+/* One launch of the register-sharing one-shot allreduce (8 ranks, bf16, all destinations per thread, launched
+ * as nuna_allreduce_oneshot launches it for `flags`: NUNA_LAUNCH_PDL, NUNA_HINT_RESIDENT; tile size and prefetch
+ * as the options say) on `stream`, in which thread 0 of block b < NUNA_DEBUG_TRACE_BLOCKS also writes to device
+ * memory trace[(slot * NUNA_DEBUG_TRACE_BLOCKS + b) * 4 + k], k = 0: global-timer ns at block start, 1: when its
+ * wait for the predecessor kernel returned, 2: when the block had issued its last store, 3: the SM it ran on.
+ * Capturable (no allocation, no synchronisation): a caller records a graph of such launches with slot = node
+ * index and reads where the time between dependent launches goes.  *grid_blocks (optional) receives the grid.  */
+#define NUNA_DEBUG_TRACE_BLOCKS 1024
+int nuna_debug_oneshot_regs_traced(const void* const* src, void* const* dst, size_t count, unsigned flags, unsigned slot,
+                                   unsigned long long* trace, unsigned* grid_blocks, void* stream);
+
 /* The probe's host-side clustering / verdict on a caller-supplied (num_sms x nlines) latency matrix.   */
 int nuna_debug_analyse_topology(const float* lat, const float* lat_rep, int num_sms, int nlines, nuna_topology_t* out);
 

@@ -66,6 +66,14 @@ __device__ __forceinline__ void prefetch_l2_bulk(const void* g, unsigned bytes)
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(g), "r"(bytes) : "memory");
 }
 
+// Nanoseconds of the device-wide timer (bounds every in-kernel wait; timestamps of the measurement aids).
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
 // ---- memory access helpers ----------------------------------------------------------------
 
 // Sources are read-only for the duration of a kernel and are re-read by other
@@ -472,13 +480,19 @@ __device__ __forceinline__ uint4 fold_vectors_own(const uint4 (&v)[N])
 // mode bit 0: streaming stores (destinations are not re-read soon); bit 1: every block asks L2 for its
 // first tile's source slices before it waits for the predecessor kernel (dependent launches with cold
 // sources only: without a predecessor there is nothing to overlap with).
-template <int N, int C, int DT>
-__global__ void __launch_bounds__(kThreads, min_blocks(N))
-k_oneshot_regs(const RankPtrs p, const size_t count, const size_t ntiles, const unsigned tv, const int mode)
+// kTimed (a measurement aid): thread 0 of every block also records, in nanoseconds of the global timer, when the
+// block started, when its wait for the predecessor returned and when it had issued its last store, plus the SM
+// it ran on: trace[(slot * trace_blocks + blockIdx.x) * 4 + {0, 1, 2, 3}] for blockIdx.x < trace_blocks.
+template <int N, int C, int DT, bool kTimed>
+__device__ __forceinline__ void oneshot_regs_body(const RankPtrs& p, const size_t count, const size_t ntiles, const unsigned tv,
+                                                  const int mode, unsigned long long* trace, const unsigned slot,
+                                                  const unsigned trace_blocks)
 {
     constexpr int kSplit = (N + C - 1) / C;
     const size_t nvec = count / Elem<DT>::kElems;
     const size_t nitems = ntiles * kSplit;
+    unsigned long long t_in = 0, t_wait = 0;
+    if (kTimed && threadIdx.x == 0) t_in = globaltimer_ns();
     if ((mode & 2) && blockIdx.x < nitems && threadIdx.x < N) {
         const size_t i0 = ((size_t)blockIdx.x / kSplit) * tv;        // thread r fetches source r's slice
         const uint4* a = p.src[0];
@@ -487,6 +501,7 @@ k_oneshot_regs(const RankPtrs p, const size_t count, const size_t ntiles, const 
         if (i0 < nvec) prefetch_l2_bulk(a + i0, (unsigned)(nvec - i0 < (size_t)tv ? nvec - i0 : (size_t)tv) * 16u);
     }
     pdl_wait();
+    if (kTimed && threadIdx.x == 0) t_wait = globaltimer_ns();
     const int stream_stores = mode & 1;
     for (size_t item = blockIdx.x; item < nitems; item += gridDim.x) {
         const size_t i = (item / kSplit) * tv + threadIdx.x;
@@ -506,6 +521,15 @@ k_oneshot_regs(const RankPtrs p, const size_t count, const size_t ntiles, const 
         }
     }
     pdl_trigger();
+    if (kTimed) {
+        __syncthreads();                                              // every warp of the block has issued its stores
+        if (threadIdx.x == 0 && blockIdx.x < trace_blocks) {
+            unsigned sm;
+            asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+            unsigned long long* o = trace + ((size_t)slot * trace_blocks + blockIdx.x) * 4;
+            o[0] = t_in; o[1] = t_wait; o[2] = globaltimer_ns(); o[3] = sm;
+        }
+    }
     const size_t tail0 = nvec * Elem<DT>::kElems;
     if (tail0 < count) {
         for (int d = blockIdx.x; d < N; d += gridDim.x) {
@@ -513,6 +537,21 @@ k_oneshot_regs(const RankPtrs p, const size_t count, const size_t ntiles, const 
             if (e < count) store_elem<DT>(p.dst[d], e, fold_scalar<N, DT>(p, e));
         }
     }
+}
+
+template <int N, int C, int DT>
+__global__ void __launch_bounds__(kThreads, min_blocks(N))
+k_oneshot_regs(const RankPtrs p, const size_t count, const size_t ntiles, const unsigned tv, const int mode)
+{
+    oneshot_regs_body<N, C, DT, false>(p, count, ntiles, tv, mode, nullptr, 0u, 0u);
+}
+
+template <int N, int C, int DT>
+__global__ void __launch_bounds__(kThreads, min_blocks(N))
+k_oneshot_regs_timed(const RankPtrs p, const size_t count, const size_t ntiles, const unsigned tv, const int mode,
+                     unsigned long long* trace, const unsigned slot, const unsigned trace_blocks)
+{
+    oneshot_regs_body<N, C, DT, true>(p, count, ntiles, tv, mode, trace, slot, trace_blocks);
 }
 
 // ---- one-shot allreduce, co-located group staged through shared memory ---------------------------------
@@ -553,13 +592,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity)
     asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                  : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return done != 0;
-}
-
-__device__ __forceinline__ unsigned long long globaltimer_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
 }
 
 // Bounded wait for phase `parity` of an mbarrier: after timeout_ns the thread latches NUNA_ERR_TIMEOUT in

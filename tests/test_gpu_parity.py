@@ -359,6 +359,34 @@ def test_graph_replay_gives_same_bits():
             assert np.array_equal(t.cpu().numpy().view(np.uint16), want)
 
 
+def test_traced_launch_matches_oracle_and_orders_its_timestamps():
+    """The measurement aid that timestamps every block of the register-sharing one-shot: the destinations still
+    receive the oracle's bits, every block reports start <= wait-return <= end on an SM that exists, and a launch
+    behind a predecessor never returns from its wait before that predecessor's last block has issued its stores."""
+    w = workloads.config_decode_activation()
+    src = workloads.make(w)
+    want = oracle.allreduce(src, nthreads=4)[0]
+    dsrc = upload(src)
+    nodes, TB = 6, nb.DEBUG_TRACE_BLOCKS
+    for flags in (0, nb.NUNA_LAUNCH_PDL, nb.NUNA_LAUNCH_PDL | nb.NUNA_HINT_RESIDENT):
+        dst = [torch.zeros(w.count, dtype=torch.int16, device="cuda") for _ in range(w.nranks)]
+        trace = torch.zeros(nodes * TB * 4, dtype=torch.int64, device="cuda")
+        grid = 0
+        for i in range(nodes):
+            grid = nb.debug_oneshot_regs_traced(dsrc, dst, w.count, flags, i, trace)
+        torch.cuda.synchronize()
+        for t in dst:
+            assert np.array_equal(t.cpu().numpy().view(np.uint16), want)
+        assert 0 < grid <= TB
+        t = trace.cpu().numpy().reshape(nodes, TB, 4)[:, :grid]
+        assert (t[:, :, 0] > 0).all() and (t[:, :, 0] <= t[:, :, 1]).all() and (t[:, :, 1] <= t[:, :, 2]).all()
+        assert (t[:, :, 3] >= 0).all() and (t[:, :, 3] < torch.cuda.get_device_properties(0).multi_processor_count).all()
+        for i in range(1, nodes):                                   # 32 ns = the timer's resolution
+            assert t[i, :, 1].min() + 32 >= t[i - 1, :, 2].max(), f"flags={flags}: node {i} passed its wait early"
+        assert (t[:, grid:, :] == 0).all() if grid < TB else True
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
 def test_headline_launch_configuration_matches_oracle():
     """The configuration the benchmark times: 8 x 512 KiB, placement AUTO with dependent launches, as nodes of one
     CUDA graph rotating over buffer sets (distinct data in each), replayed.  Every destination of every set is
