@@ -121,7 +121,7 @@ typedef enum { NUNA_BF16 = 0, NUNA_F16 = 1, NUNA_F32 = 2 } nuna_dtype_t;   /* el
  * buffer sets, at most 4 MiB per rank, else NUNA_ERR_INVALID_ARG), or always as a CUDA graph of one kernel
  * per node (NUNA_CHAIN_GRAPH).  With neither bit the library picks by measurement, which on B200 means the
  * graph at every size: the single kernel's node (two dependent memory round trips on one cluster's SMs)
- * costs 1.45 us at 16 KiB per rank against 1.15 us for a graph node launched behind its predecessor.    */
+ * costs 1.45 us at 16 KiB per rank against 1.08 us for a graph node launched behind its predecessor.    */
 #define NUNA_CHAIN_PERSISTENT 2048u
 #define NUNA_CHAIN_GRAPH      4096u
 /* `flags`, bit 13, flag-synchronised two-shot only: publish and poll the ready flags with system-scope

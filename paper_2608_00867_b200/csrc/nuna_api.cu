@@ -819,7 +819,7 @@ int launch_alltoall(Context* c, const RankPtrs& p, int nranks, size_t block_byte
 // ---- single-kernel chain ---------------------------------------------------------------------------------
 
 // One cluster runs the whole chain.  Measured on B200 (160 nodes, 8 ranks): 1.45 us per node at 16 KiB per rank
-// against 1.13-1.15 us for the graph with dependent launch, 2.5 against 1.3 us at 128 KiB, 12 against 2.5 us at
+// against 1.08 us for the graph with dependent launch, 2.5 against 1.15 us at 128 KiB, 12 against 2.4 us at
 // 1 MiB: a node still costs two dependent memory round trips (loads; then the stores the cluster barrier has to
 // see performed) plus the barrier on sixteen SMs, which is no less than a launch hidden behind its predecessor.
 // So the library never picks it by itself (limit 0); NUNA_CHAIN_PERSISTENT runs it on request.
