@@ -313,8 +313,8 @@ int nuna_allreduce_twoshot(const void* const* src, void* const* dst, int nranks,
  * choice between routing schemes by a size threshold (Section 4.1.2): one-shot while the message is small
  * enough for its single step to win (measured: up to 1 MiB per rank at 2 ranks, 512 KiB at 4, 128 KiB at
  * 8, 64 KiB at 16; under NUNA_PLACE_AUTO, whose one-shot kernel shares each tile's loads between the
- * destinations, 8 MiB of sources in total with NUNA_LAUNCH_PDL and 2 MiB without, a quarter of that beyond
- * 8 ranks; and again from 8 MiB per rank at 8 ranks or fewer, cold), beyond that the put form of the two-shot.
+ * destinations, 8 MiB of sources in total with NUNA_LAUNCH_PDL, without it 2 MiB (512 KiB beyond 8 ranks);
+ * and again from 8 MiB per rank at 8 ranks or fewer, cold), beyond that the put form of the two-shot.
  * With NUNA_TWOSHOT_SYNC the large-message choice is the flag-synchronised two-shot instead, from eight
  * times those sizes (below, the one-shot is faster than it).  Same bits whichever is chosen.            */
 int nuna_allreduce(const void* const* src, void* const* dst, int nranks,

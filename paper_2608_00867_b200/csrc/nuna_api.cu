@@ -520,14 +520,17 @@ static int launch_group(Context* c, const Options& o, const RankPtrs& p, size_t 
 // with tiles of 56 ... 256 vectors (512 KiB cold behind a dependent launch: 586 blocks of 56 vectors, 2.1 us
 // against 2.8 us with 256 full tiles); full tiles beyond.  Tiles never exceed a block's width: contiguous
 // chunks of several rows per block were slower from 8 MiB per rank (23.0 against 21.7 us).
-static unsigned regs_tile_vecs(const Context* c, const Options& o, size_t nvec, int ksplit)
+// `resident` = blocks of the kernel an SM holds: the blocks must fit in one wave (16 ranks, 3 blocks per SM, 256 KiB
+// per rank: 3.46 us with 586 blocks of 56 vectors, 2.42 us with 294 of 112).
+static unsigned regs_tile_vecs(const Context* c, const Options& o, size_t nvec, int ksplit, int resident)
 {
     if (o.regs_vecs > 0) return (unsigned)std::min(kThreads, std::max(8, o.regs_vecs / 8 * 8));
     const size_t units = nvec * (size_t)ksplit;
     const size_t one = ceil_div(ceil_div(units, (size_t)c->num_sms), (size_t)8) * 8;
     if (one <= 56) return (unsigned)std::max<size_t>(8, one);
-    const size_t four = ceil_div(ceil_div(units, (size_t)c->num_sms * 4), (size_t)8) * 8;
-    return (unsigned)std::min<size_t>(kThreads, std::max<size_t>(56, four));
+    const size_t per_sm = (size_t)std::max(1, std::min(4, resident));
+    const size_t many = ceil_div(ceil_div(units, (size_t)c->num_sms * per_sm), (size_t)8) * 8;
+    return (unsigned)std::min<size_t>(kThreads, std::max<size_t>(56, many));
 }
 
 template <int N, int C, int DT>
@@ -537,7 +540,7 @@ static int launch_regs(Context* c, const Options& o, const RankPtrs& p, size_t c
     auto k = k_oneshot_regs<N, C, DT>;
     constexpr int kSplit = (N + C - 1) / C;
     const size_t nvec = count / Elem<DT>::kElems;
-    const unsigned tv = regs_tile_vecs(c, o, nvec, kSplit);
+    const unsigned tv = regs_tile_vecs(c, o, nvec, kSplit, NUNA_OCC(k));
     const size_t ntiles = ceil_div(nvec, (size_t)tv);
     const size_t nitems = std::max<size_t>(ntiles * kSplit, (count % Elem<DT>::kElems) ? (size_t)N : 0);
     const unsigned grid = pick_grid(c, o, std::max<size_t>(nitems, 1), NUNA_OCC(k), 0);
@@ -957,14 +960,15 @@ int nuna_allreduce(const void* const* src, void* const* dst, int nranks, size_t 
     // with NUNA_PLACE_AUTO the one-shot side is the register-sharing kernel, which stays ahead of the put form up
     // to 8 MiB of sources in total behind a dependent launch (8 ranks, cold: 128 KiB 1.51 vs 1.92 us, 1 MiB 3.33 vs
     // 3.74, 2 MiB 6.44 vs 6.16; 4 ranks: 2 MiB 3.34 vs 3.52, 4 MiB 5.79 vs 5.73) and up to 2 MiB launched plainly
-    // (8 ranks: 256 KiB 2.65 vs 2.70, 512 KiB 3.29 vs 3.17); beyond 8 ranks, where it needs two passes over the
-    // sources, a quarter of that (16 ranks: 64 KiB 1.68 vs 2.69, 256 KiB 3.49 vs 3.25)
+    // (8 ranks: 256 KiB 2.65 vs 2.70, 512 KiB 3.29 vs 3.17; beyond 8 ranks, where it needs two passes over the
+    // sources, a quarter of that); 16 ranks behind a dependent launch: 256 KiB 2.33 vs 3.21, 512 KiB 3.52 vs 4.25,
+    // 1 MiB 7.3 vs 6.6
     // From 8 MiB per rank at 8 ranks or fewer it is ahead again, with two blocks per tile (8 ranks: 8 MiB 21.3 vs 21.6 us,
     // 16 MiB 41.2 vs 42.1, 64 MiB 157.7 vs 160.8).
     bool oneshot_large = false;
     if ((flags & NUNA_PLACE_MASK) == NUNA_PLACE_AUTO) {
         const size_t total = (flags & NUNA_LAUNCH_PDL) ? (size_t)8 << 20 : (size_t)2 << 20;
-        limit = std::max(limit, (nranks <= 8 ? total : total / 4) / (size_t)nranks);
+        limit = std::max(limit, ((nranks <= 8 || (flags & NUNA_LAUNCH_PDL)) ? total : total / 4) / (size_t)nranks);
         oneshot_large = nranks <= 8 && bytes >= ((size_t)8 << 20) && !(flags & NUNA_HINT_RESIDENT);
     }
     constexpr size_t kSyncFactor = 8;
@@ -1260,7 +1264,7 @@ int nuna_debug_oneshot_regs_traced(const void* const* src, void* const* dst, siz
     const Options o = snapshot(c);
     auto k = k_oneshot_regs_timed<N, 8, kBf16>;
     const size_t nvec = count / 8;
-    const unsigned tv = regs_tile_vecs(c, o, nvec, 1);
+    const unsigned tv = regs_tile_vecs(c, o, nvec, 1, NUNA_OCC(k));
     const size_t ntiles = ceil_div(nvec, (size_t)tv);
     const size_t nitems = std::max<size_t>(ntiles, (count % 8) ? (size_t)N : 0);
     const unsigned grid = pick_grid(c, o, std::max<size_t>(nitems, 1), NUNA_OCC(k), 0);
