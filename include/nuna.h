@@ -265,7 +265,7 @@ int nuna_init(size_t scratch_bytes);
  *                           Section 6.5: few blocks vs many)
  *  NUNA_OPT_UNROLL          vectors per thread per work item (1, 2, 4; limited so that N * unroll <= 16)
  *  NUNA_OPT_COLOC           destinations of a tile that share a block (co-located group, work lists) or a thread
- *                           (NUNA_PLACE_REGS) in the placement-aware one-shot (2, 4, 8; 0 = by rank count and hint)
+ *                           (NUNA_PLACE_REGS; also 16 beyond 8 ranks) in the placement-aware one-shot (2, 4, 8; 0 = by rank count and hint)
  *  NUNA_OPT_AUTO_MIN_BYTES  NUNA_PLACE_AUTO never picks a placement-aware kernel below this many bytes per rank
  *                           (on top of its measured crossover)
  *  NUNA_OPT_TIMEOUT_MS      limit of every in-kernel wait (ready flags, barrier, bulk-copy completion)

@@ -587,10 +587,11 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
     else if (place == NUNA_PLACE_AUTO) which = auto_kernel(c, o, nranks, bytes, flags);
     if (which == OneShotKernel::Regs) {
         const unsigned m = (flags & NUNA_LAUNCH_PDL) ? kLaunchPdl : kLaunchPlain;
-        // destinations per thread: all of them (eight at most), so that a tile crosses the L2 -> SM fabric once;
-        // half of them for large cold messages, where two blocks per tile keep more DRAM loads in flight
-        // (8 ranks x 16 MiB cold: 41.8 us with four, 42.0 with eight; 16 ranks x 4 MiB: 21.5 us with eight, 24.0 with four)
-        const int all = std::min(8, pow2_at_least(nranks));
+        // destinations per thread: all of them, so that a tile crosses the L2 -> SM fabric once (beyond 8 ranks the
+        // sixteen-destination form: 9 ranks x 512 KiB 2.25 us against 2.71 in two passes of eight, 16 ranks x 1 MiB
+        // 6.39 against 7.35); half of them for large cold messages, where two blocks per tile keep more DRAM loads
+        // in flight (8 ranks x 16 MiB cold: 41.8 us with four, 42.0 with eight)
+        const int all = nranks > 8 ? 16 : std::min(8, pow2_at_least(nranks));
         const bool large_cold = !(flags & NUNA_HINT_RESIDENT) && bytes >= ((size_t)8 << 20);
         int coloc = o.coloc > 0 ? o.coloc : (large_cold ? std::min(8, std::max(2, pow2_at_least(nranks) / 2)) : all);
         while (coloc > 2 && coloc / 2 >= nranks) coloc >>= 1;
@@ -598,6 +599,7 @@ int launch_oneshot(Context* c, const RankPtrs& p, int nranks, int dtype, size_t 
             constexpr int N = decltype(n_)::value, DT = decltype(d_)::value;
             // from 8 MiB per rank the prefetch only adds requests to a saturated memory system
             // (8 ranks, four destinations per thread: 16 MiB 45.5 us with, 41.2 without; 64 MiB 175 against 158)
+            if constexpr (N > 8) { if (coloc >= 16) return launch_regs<N, 16, DT>(c, o, p, count, flags, m, !large_cold, stream); }
             if (coloc >= 8) return launch_regs<N, 8, DT>(c, o, p, count, flags, m, !large_cold, stream);
             if (coloc >= 4) return launch_regs<N, 4, DT>(c, o, p, count, flags, m, !large_cold, stream);
             return launch_regs<N, 2, DT>(c, o, p, count, flags, m, !large_cold, stream);
