@@ -523,6 +523,8 @@ def run_gpu(args):
         # latency-bound kernels read 30-50 % slower than in a fresh process, 140-180 against 95 us at 8 blocks.)
         blocks_rows = {}
         for label, fn_of in (("oneshot_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_oneshot(s, d, c1, stream=st))),
+                             ("oneshot_auto_resident_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_oneshot(
+                                 s, d, c1, flags=nb.NUNA_PLACE_AUTO | nb.NUNA_HINT_RESIDENT, stream=st))),
                              ("twoshot_put_1MiB", lambda: (lambda s, d, st: nb.nuna_allreduce_twoshot(s, d, c1, flags=nb.NUNA_TWOSHOT_PUT, stream=st)))):
             row = {}
             for blocks in (8, 37, 148, 592, 0):

@@ -526,9 +526,13 @@ static unsigned regs_tile_vecs(const Context* c, const Options& o, size_t nvec, 
 {
     if (o.regs_vecs > 0) return (unsigned)std::min(kThreads, std::max(8, o.regs_vecs / 8 * 8));
     const size_t units = nvec * (size_t)ksplit;
+    const size_t per_sm = (size_t)std::max(1, std::min(4, resident));
+    if (o.blocks > 0 && (size_t)o.blocks < (size_t)c->num_sms * per_sm) {          // a capped grid: as few tiles as blocks, then full tiles
+        const size_t capped = ceil_div(ceil_div(units, (size_t)o.blocks), (size_t)8) * 8;
+        return (unsigned)std::min<size_t>(kThreads, std::max<size_t>(8, capped));
+    }
     const size_t one = ceil_div(ceil_div(units, (size_t)c->num_sms), (size_t)8) * 8;
     if (one <= 56) return (unsigned)std::max<size_t>(8, one);
-    const size_t per_sm = (size_t)std::max(1, std::min(4, resident));
     const size_t many = ceil_div(ceil_div(units, (size_t)c->num_sms * per_sm), (size_t)8) * 8;
     return (unsigned)std::min<size_t>(kThreads, std::max<size_t>(56, many));
 }

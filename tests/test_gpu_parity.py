@@ -141,9 +141,18 @@ def test_register_oneshot_tile_sizes_and_prefetch(vecs, n):
                 nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=flags)
                 for got in dst.numpy():
                     assert_same_bits(got, want, f"regs vecs={vecs} n={n} count={count} flags={flags} nopf={no_prefetch}")
+            if vecs == 0:                                            # a capped grid: blocks loop over several tiles
+                for blocks in (1, 5, 37):
+                    nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, blocks)
+                    dst = Dst(n, count)
+                    nb.nuna_allreduce_oneshot(dsrc, dst.view, count, flags=base | nb.NUNA_LAUNCH_PDL)
+                    for got in dst.numpy():
+                        assert_same_bits(got, want, f"regs blocks={blocks} n={n} count={count}")
+                nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, 0)
     finally:
         nb.nuna_set_option(nb.NUNA_OPT_REGS_VECS, 0)
         nb.nuna_set_option(nb.NUNA_OPT_PREFETCH, 0)
+        nb.nuna_set_option(nb.NUNA_OPT_BLOCKS, 0)
     assert nb.nuna_device_status() == nb.NUNA_OK
 
 
