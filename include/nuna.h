@@ -274,10 +274,11 @@ int nuna_init(size_t scratch_bytes);
  *                           more = every probed domain cut into equal latency quantiles; 0 = what the probe found
  *  NUNA_OPT_STAGE_VECS      16-byte vectors per source per tile of the NUNA_PLACE_STAGED kernel (0 = by size)
  *  NUNA_OPT_TWOSHOT_VECS    16-byte vectors per tile (= per ready flag) of the flag-synchronised two-shot (0 = by size)
- *  NUNA_OPT_AG_BULK_VECS    nuna_allgather / nuna_alltoall move their (rank, tile) work items through the bulk-copy
- *                           engine (one bulk load into shared memory, one bulk store per destination) by default (0,
- *                           tile size by message size); >= 8: tiles of that many 16-byte vectors; 1: the register
- *                           form instead (16-byte loads and stores by every thread)
+ *  NUNA_OPT_AG_BULK_VECS    0 (default): nuna_allgather uses 16-byte loads and stores on small tiles up to 128 MiB of
+ *                           output and, like nuna_alltoall at every size, the bulk-copy engine beyond (one bulk load
+ *                           into shared memory, one bulk store per destination; tile size by message size);
+ *                           >= 8: the bulk-copy form with tiles of that many 16-byte vectors; 1: the register form
+ *                           with full tiles (16-byte loads and stores by every thread)
  *  NUNA_OPT_REGS_VECS       16-byte vectors per source per tile of the NUNA_PLACE_REGS kernel (8 ... 256; 0 = by size)
  *  NUNA_OPT_PREFETCH        1: kernels launched with NUNA_LAUNCH_PDL do not ask L2 for their first tile ahead of the
  *                           wait for their predecessor (0 = they do, unless NUNA_HINT_RESIDENT is given); a

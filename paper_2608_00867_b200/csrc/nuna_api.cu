@@ -771,6 +771,17 @@ int launch_allgather(Context* c, const RankPtrs& p, int nranks, size_t shard_byt
         return launch(k_allgather_scalar, grid, stream, mode, p, nranks, shard16);
     }
     const size_t shard_vec = shard_bytes / 16;
+    const size_t out_total = shard_bytes * (size_t)nranks * (size_t)nranks;
+    if (o.ag_bulk_vecs == 0 && out_total <= ((size_t)128 << 20)) {
+        // register form with small tiles: about four blocks per SM, tiles of 16 ... 256 vectors
+        const size_t per = ceil_div(ceil_div(shard_vec * (size_t)nranks, (size_t)c->num_sms * 4), (size_t)8) * 8;
+        const unsigned tv = (unsigned)std::min<size_t>(kThreads, std::max<size_t>(16, per));
+        const size_t tiles = ceil_div(shard_vec, (size_t)tv);
+        const unsigned grid = (unsigned)(tiles * nranks);
+        if (o.blocks <= 0 || (size_t)o.blocks >= grid)             // one tile per block: a capped grid takes the looping form below
+            return launch(k_allgather_small, grid, stream, mode, p, nranks, shard_vec, tiles, tv,
+                          prefetch_pays(o, flags, nranks, shard_vec * 16) ? 1 : 0);
+    }
     if (o.ag_bulk_vecs != 1) {
         // Default: the bulk-copy form, one block per (rank, tile); the copy engine moves the tile in once and
         // out N times.  Measured against the register form below: 16 x 64 KiB 4.11 vs 4.99 us, 16 x 8 KiB 2.02

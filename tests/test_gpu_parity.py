@@ -260,6 +260,23 @@ def test_allgather_and_alltoall_copy_forms(bulk_vecs):
     assert nb.nuna_device_status() == nb.NUNA_OK
 
 
+def test_allgather_large_output_takes_the_bulk_copy_form_by_default():
+    """Beyond 128 MiB of output the default allgather is the bulk-copy form with its size-chosen tile: 8 ranks x 5 MiB
+    + 16 bytes (a ragged last tile), raw bits, every destination compared in full on the device."""
+    n, shard = 8, 5 * 512 * 1024 + 8
+    g = torch.Generator(device="cuda")
+    g.manual_seed(99)
+    src = [torch.randint(-32768, 32767, (shard,), generator=g, device="cuda", dtype=torch.int16) for _ in range(n)]
+    dst = [torch.full((n * shard,), -1, dtype=torch.int16, device="cuda") for _ in range(n)]
+    nb.nuna_allgather(src, dst, shard, flags=nb.NUNA_LAUNCH_PDL)
+    torch.cuda.synchronize()
+    want = oracle.allgather([x.cpu().numpy().view(np.uint16) for x in src])[0]
+    assert np.array_equal(dst[0].cpu().numpy().view(np.uint16), want)
+    for d in dst[1:]:
+        assert torch.equal(d, dst[0])                                # all destinations identical
+    assert nb.nuna_device_status() == nb.NUNA_OK
+
+
 def test_config_allgather16_raw_bits():
     w = workloads.config_allgather16()
     rng = np.random.Generator(np.random.PCG64(w.seed))
