@@ -402,7 +402,13 @@ def run_gpu(args):
     empty_pdl = lambda s, d, st: nb.nuna_launch_floor(grid_blocks, flags=nb.NUNA_LAUNCH_PDL, stream=st)
     floor_us = per_call_us(empty, sets, 1000)
     floor_pdl_us = per_call_us(empty_pdl, sets, 1000)
+    # the same empty kernel releasing its successor before its own wait, and with a single block: how closely
+    # graph nodes can follow one another at all
+    floor_first_us = per_call_us(lambda s, d, st: nb.debug_launch_floor(grid_blocks, nb.NUNA_LAUNCH_PDL, True, st), sets, 1000)
+    floor_one_us = per_call_us(lambda s, d, st: nb.nuna_launch_floor(1, flags=nb.NUNA_LAUNCH_PDL, stream=st), sets, 1000)
     floors = {"graph_node_us": round(floor_us, 3), "graph_node_pdl_us": round(floor_pdl_us, 3),
+              "graph_node_pdl_trigger_first_us": round(floor_first_us, 3),
+              "graph_node_pdl_one_block_us": round(floor_one_us, 3),
               "eager_event_pair_us": isolated_stats(empty, sets),
               "eager_launch_plus_stream_sync_host_us": host_sync_floor(empty, sets),
               "grid_blocks": grid_blocks}

@@ -160,6 +160,8 @@ def lib() -> ctypes.CDLL:
         L.nuna_debug_oneshot_regs_traced.argtypes = [vpp, vpp, ctypes.c_size_t, ctypes.c_uint, ctypes.c_uint, ctypes.c_void_p,
                                                      ctypes.POINTER(ctypes.c_uint), ctypes.c_void_p]
         L.nuna_debug_oneshot_regs_traced.restype = ctypes.c_int
+        L.nuna_debug_launch_floor.argtypes = [ctypes.c_uint, ctypes.c_uint, ctypes.c_int, ctypes.c_void_p]
+        L.nuna_debug_launch_floor.restype = ctypes.c_int
         L.nuna_debug_twoshot.argtypes = [vpp, vpp, ctypes.c_int, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint, ctypes.c_uint]
         L.nuna_debug_twoshot.restype = ctypes.c_int
         _lib = L
@@ -366,6 +368,11 @@ def nuna_device_status() -> int:
 
 def nuna_launch_floor(blocks: int, flags: int = 0, stream=None, check: bool = True) -> int:
     return _finish(lib().nuna_launch_floor(blocks, flags, _stream(stream)), "nuna_launch_floor", check)
+
+
+def debug_launch_floor(blocks: int, flags: int = 0, trigger_first: bool = False, stream=None) -> int:
+    return _finish(lib().nuna_debug_launch_floor(blocks, flags, 1 if trigger_first else 0, _stream(stream)),
+                   "nuna_debug_launch_floor", True)
 
 
 def nuna_launch_count() -> int:

@@ -1142,6 +1142,13 @@ int nuna_launch_floor(unsigned blocks, unsigned flags, void* stream)
     return launch(k_empty, blocks, (cudaStream_t)stream, launch_mode(flags), 0);
 }
 
+// See nuna_debug.h.
+int nuna_debug_launch_floor(unsigned blocks, unsigned flags, int trigger_first, void* stream)
+{
+    if (blocks == 0 || blocks > (1u << 20) || (flags & ~NUNA_LAUNCH_PDL)) return NUNA_ERR_INVALID_ARG;
+    return launch(k_empty, blocks, (cudaStream_t)stream, launch_mode(flags), trigger_first ? 1 : 0);
+}
+
 unsigned long long nuna_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* nuna_status_string(int status)

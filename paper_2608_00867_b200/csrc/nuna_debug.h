@@ -50,6 +50,10 @@ int nuna_debug_access_latency(const void* const* src, void* const* dst, size_t c
 int nuna_debug_oneshot_regs_traced(const void* const* src, void* const* dst, size_t count, unsigned flags, unsigned slot,
                                    unsigned long long* trace, unsigned* grid_blocks, void* stream);
 
+/* nuna_launch_floor's empty kernel; with trigger_first != 0 it releases its dependent launch before it waits
+ * for its own predecessor instead of after.                                                              */
+int nuna_debug_launch_floor(unsigned blocks, unsigned flags, int trigger_first, void* stream);
+
 /* The probe's host-side clustering / verdict on a caller-supplied (num_sms x nlines) latency matrix.   */
 int nuna_debug_analyse_topology(const float* lat, const float* lat_rep, int num_sms, int nlines, nuna_topology_t* out);
 

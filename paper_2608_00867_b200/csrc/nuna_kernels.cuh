@@ -1491,6 +1491,14 @@ __global__ void k_barrier_selftest(BarrierWords* bw, unsigned int expected, unsi
 }
 
 // Launch-floor reference: same grid shape, no memory traffic.
-__global__ void __launch_bounds__(kThreads) k_empty(int) { pdl_wait(); pdl_trigger(); }
+// The launch floor: waits for its predecessor and lets its successor go, like every collective kernel.
+// trigger_first = 1 releases the successor before waiting (a measurement aid: how closely launches can follow
+// one another when nothing delays the trigger).
+__global__ void __launch_bounds__(kThreads) k_empty(int trigger_first)
+{
+    if (trigger_first) pdl_trigger();
+    pdl_wait();
+    pdl_trigger();
+}
 
 }  // namespace nuna
