@@ -1146,7 +1146,8 @@ int nuna_launch_floor(unsigned blocks, unsigned flags, void* stream)
 int nuna_debug_launch_floor(unsigned blocks, unsigned flags, int trigger_first, void* stream)
 {
     if (blocks == 0 || blocks > (1u << 20) || (flags & ~NUNA_LAUNCH_PDL)) return NUNA_ERR_INVALID_ARG;
-    return launch(k_empty, blocks, (cudaStream_t)stream, launch_mode(flags), trigger_first ? 1 : 0);
+    if (trigger_first) return launch(k_empty_trigger_first, blocks, (cudaStream_t)stream, launch_mode(flags), 0);
+    return launch(k_empty, blocks, (cudaStream_t)stream, launch_mode(flags), 0);
 }
 
 unsigned long long nuna_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
