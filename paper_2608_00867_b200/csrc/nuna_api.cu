@@ -660,22 +660,27 @@ int launch_twoshot_flags(int num_sms, int blocks_override, const RankPtrs& p, in
 {
     const size_t bytes = count * elem_size(dtype);
     const size_t nvec = count / elems_per_vec(dtype);
+    bool mid_sized = false;
     if (tv == 0) {
         // Tile bytes across all N sources, from a sweep at 8 ranks (16 ... 256 vectors per tile at every size):
         // small tiles while the message is small (more blocks, less latency per tile), 32 KiB once there are
         // plenty.  At 8 MiB of sources 16 KiB tiles make 1024 blocks for 592 resident ones and the second
         // wave's consumers wait (10.3 us against 7.6 us with 12 KiB tiles), hence the step back there.
+        // Between 16 and 64 MiB of sources 24 KiB tiles with a lead of five blocks per SM are ahead (3 MiB per rank 11.6
+        // against 12.3 us, 4 MiB 14.2 against 15.1, 6 MiB 19.1 against 21.3, 7 MiB 21.6 against 24.2; at 8 MiB 27.2
+        // against 24.8, hence the upper limit).
         const size_t src_bytes = bytes * (size_t)nranks;
+        mid_sized = nranks <= 8 && src_bytes > ((size_t)16 << 20) && src_bytes < ((size_t)64 << 20);   // 16 ranks: no gain
         const unsigned tile_src = src_bytes <= ((size_t)512 << 10) ? 4096u : src_bytes <= ((size_t)1 << 20) ? 8192u
                                 : src_bytes <= ((size_t)8 << 20) ? 12288u
-                                : src_bytes <= ((size_t)32 << 20) ? 16384u : 32768u;
+                                : src_bytes <= ((size_t)16 << 20) ? 16384u : mid_sized ? 24576u : 32768u;
         tv = tile_src / 16u / (unsigned)nranks;
     }
     tv = std::max(min_tv, std::min(tv, 2048u / (unsigned)nranks));
     tv = std::max(1u, tv / 8u * 8u);
     if (tv < min_tv) tv = min_tv;
     const size_t ntiles = std::max<size_t>(1, ceil_div(nvec, (size_t)tv));
-    unsigned lead_max = (unsigned)num_sms * 8u;
+    unsigned lead_max = (unsigned)num_sms * (mid_sized ? 5u : 8u);
     if (blocks_override > 0) lead_max = (unsigned)std::max(1, blocks_override);
     const size_t lead = std::min<size_t>(ntiles, lead_max);
     const unsigned grid = (unsigned)(ntiles + lead);
